@@ -1,0 +1,288 @@
+/*
+ * cascade.h -- C ABI of the B200 (sm_100a) tree-verification library for CASCADE
+ * ("CASCADE: Context-Aware Relaxation for Speculative Image Decoding").
+ *
+ * One verification step of tree-based speculative image decoding: the target model looks at a draft
+ * token tree in one pass (Section 3, "tree decoding"), and the relaxed acceptance rule of Section 4
+ * (Eq. 1-3, Algorithm 2) decides which root-to-node path of draft tokens is kept.
+ *
+ * Conventions
+ *   - Every function returns an int status: CASCADE_OK (0) or a negative CASCADE_ERR_* code.  Nothing
+ *     throws or aborts.  All arguments are validated on the host before anything is launched, so a bad
+ *     argument never reaches the device.
+ *   - Pointers are DEVICE pointers unless the parameter is documented "host".  The caller owns every
+ *     data buffer; the library owns only what cascade_create / cascade_tree_create return, until the
+ *     matching destroy call.
+ *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = default stream)
+ *     and is asynchronous: outputs are valid after the stream has been synchronised.
+ *   - A context is bound to the device that was current at cascade_create and holds scratch memory
+ *     that its calls share: calls on ONE context must not overlap on the GPU (use one stream, or one
+ *     context per stream).
+ *   - Tensors are dense, row-major, innermost index last.  "elem" is the context's dtype
+ *     (float for CASCADE_F32, bf16 bit patterns for CASCADE_BF16).
+ *   - Notation: B prompts; R = 2B rows of the classifier-free-guidance pair, cond rows 0..B-1 then
+ *     uncond rows B..2B-1; T tree rows INCLUDING the root row 0 (the pending, last-emitted token whose
+ *     key/value is not yet in the cache); P prefix (KV cache) length; h hidden size; Hq/Hkv query/kv
+ *     heads; D head size; V image-token vocabulary.
+ */
+#ifndef CASCADE_H_
+#define CASCADE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------------------------------ */
+#define CASCADE_OK 0
+#define CASCADE_ERR_INVALID_ARG (-1)       /* null pointer, non-positive size, value out of range     */
+#define CASCADE_ERR_BAD_TREE (-2)          /* parent[] is not a BFS-ordered tree with grouped siblings */
+#define CASCADE_ERR_WORKSPACE (-3)         /* device allocation of the context's scratch failed        */
+#define CASCADE_ERR_UNSUPPORTED_SHAPE (-4) /* shape outside what the kernels handle (see cascade_shape) */
+#define CASCADE_ERR_CUDA (-5)              /* a CUDA runtime / driver call failed                      */
+#define CASCADE_ERR_TIMEOUT (-6)           /* a bounded device-side wait gave up (see cascade_check)   */
+
+/* ---- enums ------------------------------------------------------------------------------------- */
+#define CASCADE_F32 0
+#define CASCADE_BF16 1
+
+/* cascade_params.flags */
+#define CASCADE_USE_I 1u          /* Eq. 1: add the mass of interchangeable siblings                     */
+#define CASCADE_USE_C 2u          /* Eq. 2: add the mass of convergent children                          */
+#define CASCADE_CONV_DIST_SELF 4u /* Eq. 3 read literally: a child's mass is taken under the candidate's
+                                     own row; default (flag clear) follows Algorithm 2, which reads it
+                                     from the same distribution as the candidate's own probability       */
+
+/* cascade_select_path mode */
+#define CASCADE_SELECT_LONGEST 0      /* deepest node whose whole path is accepted, smallest index first */
+#define CASCADE_SELECT_FIRST_ACCEPT 1 /* Algorithm 2's walk: first accepted child at every level         */
+
+/* A score this close to its threshold is counted in near_count (decisions there are not stable under
+ * rounding). */
+#define CASCADE_NEAR 1e-3f
+
+#define CASCADE_MAX_TREE_ROWS 256   /* T  <= 256                                            */
+#define CASCADE_MAX_CHILDREN 32     /* children of one node <= 32                           */
+
+typedef struct cascade_ctx cascade_ctx;
+typedef struct cascade_tree cascade_tree;
+
+/* Fixed sizes of a context.  Supported: D in {64,128}; Hq a multiple of Hkv; h a multiple of 64;
+ * V a multiple of 8; T_max <= CASCADE_MAX_TREE_ROWS; B >= 1.  ffn may be 0 if no decoder layer is
+ * run through cascade_verify_step (otherwise a multiple of 64). */
+typedef struct {
+  int32_t dtype; /* CASCADE_F32 or CASCADE_BF16: element type of q/k/v, hidden states and weights */
+  int32_t B;
+  int32_t T_max;
+  int32_t P_max; /* largest prefix length any call will use                                      */
+  int32_t h, Hq, Hkv, D, V;
+  int32_t ffn;
+} cascade_shape;
+
+/* Relaxation parameters (Section 4.1: tau_pos gates Eq. 1, tau_seq gates Eq. 2; Eq. 3 / Algorithm 2:
+ * tvd_budget is the total-variation budget of one verification step, 0.5 in the paper). */
+typedef struct {
+  float tau_pos;
+  float tau_seq;
+  float tvd_budget;
+  uint32_t flags; /* CASCADE_USE_I | CASCADE_USE_C [| CASCADE_CONV_DIST_SELF] */
+} cascade_params;
+
+/* ---- life cycle -------------------------------------------------------------------------------- */
+
+/* Create a context on the current device and allocate its scratch (split-KV partial results,
+ * activation staging, softmax partials).  *out is set only on success. */
+int cascade_create(cascade_ctx** out, const cascade_shape* shape);
+int cascade_destroy(cascade_ctx* ctx);
+
+/* Bytes of device scratch the context holds. */
+int64_t cascade_workspace_bytes(const cascade_ctx* ctx);
+
+/* Reads the context's device-side error word (set when a bounded wait inside a kernel ran out) after
+ * synchronising `stream`.  Returns CASCADE_OK, CASCADE_ERR_TIMEOUT or CASCADE_ERR_CUDA, and clears
+ * the word. */
+int cascade_check(cascade_ctx* ctx, void* stream);
+
+/* Number of kernels the most recent call on this context enqueued. */
+int cascade_last_launch_count(const cascade_ctx* ctx);
+
+const char* cascade_strerror(int status);
+
+/* The draft tree (the static tree mask of Section 3; Algorithm 2 input `tree`).
+ * parent: HOST array of T entries, parent[0] = -1, 0 <= parent[j] < j, rows in BFS order (depth never
+ * decreases with the index) and the children of one parent contiguous.  Builds the device-side
+ * descriptor: depth, packed ancestor-or-self bitmask (T x 4 uint64 words), child ranges, and the list
+ * of (node, node) pairs whose cosine the acceptance rule reads (every parent->child edge, then every
+ * unordered sibling pair).  Returns CASCADE_ERR_BAD_TREE if the ordering rules do not hold. */
+int cascade_tree_create(cascade_ctx* ctx, int32_t T, const int32_t* parent, cascade_tree** out);
+int cascade_tree_destroy(cascade_tree* tree);
+int32_t cascade_tree_rows(const cascade_tree* tree);      /* T                                     */
+int32_t cascade_tree_depth(const cascade_tree* tree);     /* deepest level                         */
+int32_t cascade_tree_num_pairs(const cascade_tree* tree); /* edges + sibling pairs                 */
+/* Copies the pair list to HOST arrays of cascade_tree_num_pairs entries (for inspecting scores). */
+int cascade_tree_pairs(const cascade_tree* tree, int32_t* pair_a, int32_t* pair_b);
+
+/* ---- (a) tree-masked attention ----------------------------------------------------------------- */
+/* Section 3: all draft-tree rows are verified by the target "via a parallel forward pass".  For every
+ * row r of the CFG pair, head and tree row j:
+ *     out[r,j,head,:] = sum_i softmax_i(softmax_scale * <q[r,j,head,:], k_i>) v_i
+ * over the keys row j may see: cache entries 0..prefix_len[r]-1 and the tree rows that are j itself or
+ * one of its ancestors.  Query head `head` reads kv head head / (Hq / Hkv).
+ *   q        [R,T,Hq,D] elem          k_tree, v_tree [R,T,Hkv,D] elem
+ *   k_prefix, v_prefix [R,prefix_cap,Hkv,D] elem; rows at or beyond prefix_len[r] are never used
+ *   prefix_len [R] int32, device; 0 <= prefix_len[r] <= min(prefix_cap, P_max)
+ *   out      [R,T,Hq,D] elem
+ * Softmax and accumulation are fp32.  Base addresses must be 16-byte aligned. */
+int cascade_tree_attn(cascade_ctx* ctx, const cascade_tree* tree, const void* q, const void* k_prefix,
+                      const void* v_prefix, int32_t prefix_cap, const int32_t* prefix_len,
+                      const void* k_tree, const void* v_tree, void* out, float softmax_scale,
+                      void* stream);
+
+/* ---- (b) final norm + LM head + classifier-free guidance + vocabulary softmax statistics ------- */
+/* Section 4.2 names the final projection, O(hV), as the dominant cost of verification; the guidance
+ * scale is the experimental setting of App. D.2 (3.0, or 5.0 for Janus-Pro).  For prompt b, tree row j:
+ *     n_x      = hidden_x * rsqrt(mean(hidden_x^2) + eps) * rms_gamma         x in {cond, uncond}
+ *     logits   = (W n_u + cfg_scale * (W n_c - W n_u)) / temperature
+ *     feat     = n_c                 (the target hidden state F of Section 4.1 that feeds the head)
+ *     row_lse  = log sum_v exp(logits[v])
+ *     cand_parent[b,j]  = logits[b, parent[j], tok[b,j]]              (0 for the root)
+ *     cand_gparent[b,j] = logits[b, parent[parent[j]], tok[b,j]]      (0 where there is none)
+ *   hidden [R,T,h] elem; rms_gamma [h] float; w_head [V,h] elem; tok [B,T] int32 in [0,V)
+ *   logits_out [B,T,V] float or NULL; feat_out [B,T,h] float; feat_norm_out [B,T] float (||feat||_2);
+ *   row_lse_out [B,T] float; cand_parent_out, cand_gparent_out [B,T] float (both NULL if tok is NULL).
+ * The guidance mix is applied to the normalised hidden states before the product (the head is
+ * linear), and that operand is carried as a bf16 high part plus a bf16 remainder so the result keeps
+ * fp32-level accuracy.  temperature > 0. */
+int cascade_lm_head_cfg(cascade_ctx* ctx, const cascade_tree* tree, const void* hidden,
+                        const float* rms_gamma, float eps, const void* w_head, float cfg_scale,
+                        float temperature, const int32_t* tok, float* logits_out, float* feat_out,
+                        float* feat_norm_out, float* row_lse_out, float* cand_parent_out,
+                        float* cand_gparent_out, void* stream);
+
+/* ---- (c) relaxed acceptance -------------------------------------------------------------------- */
+/* Cosines of Section 4.1 for the tree's pair list: scores_out[b,i] = cos(feat[b,pair_a[i]],
+ * feat[b,pair_b[i]]).  feat [B,T,feat_dim] float; feat_norm [B,T] float or NULL (then computed here).
+ * Passing logits as feat (feat_dim = V) gives the logit-space variant of App. B. */
+int cascade_similarity(cascade_ctx* ctx, const cascade_tree* tree, const float* feat, int32_t feat_dim,
+                       const float* feat_norm, float* scores_out, void* stream);
+
+/* Eq. 1-3 and Algorithm 2 for every draft node at once.  For node j >= 1 with parent pi,
+ * g = softmax(logits[b,pi,:]):
+ *     q_j  = g[tok_j]
+ *     I_j  = siblings s of j with cos(F_j,F_s) >= tau_pos ; C_j = children c of j with cos >= tau_seq
+ *     mI_j = mass under g of the distinct tokens of I_j other than tok_j
+ *     mC_j = mass (under g, or under softmax(logits[b,j,:]) with CASCADE_CONV_DIST_SELF) of the distinct
+ *            tokens of C_j not equal to tok_j and not already in mI_j
+ *     running total t: the first child of pi starts from tvd_out[pi], a later sibling from the previous
+ *     sibling's tvd_out (what Algorithm 2's curr_TVD holds when its walk arrives at j);
+ *     each set is added whole, I first, only if non-empty and t + mass <= tvd_budget;
+ *     accept[j] = uniforms[j] < min(1, q_relaxed[j] / draft_p[j]);  draft_p <= 0 rejects; accept[0] = 1.
+ * Inputs: scores [B,num_pairs] float from cascade_similarity; row_lse, cand_parent, cand_gparent [B,T]
+ * float as produced by cascade_lm_head_cfg -- or pass logits [B,T,V] float (then those three may be
+ * NULL and are derived from logits); tok [B,T] int32; draft_p [B,T] float (the drafter's probability of
+ * tok[j] under its parent's context: Algorithm 2 input D); uniforms [B,T] float in [0,1) (Algorithm 2's
+ * random(), made an input so results are reproducible).
+ * Outputs: accept [B,T] uint8; q_relaxed, tvd_out [B,T] float; near_count [B] int32 = number of nodes
+ * with a cosine, a budget comparison or the accept test within CASCADE_NEAR of its threshold (any of
+ * the last three may be NULL). */
+int cascade_relaxed_accept(cascade_ctx* ctx, const cascade_tree* tree, const float* scores,
+                           const float* logits, const float* row_lse, const float* cand_parent,
+                           const float* cand_gparent, const int32_t* tok, const float* draft_p,
+                           const float* uniforms, const cascade_params* params, uint8_t* accept,
+                           float* q_relaxed, float* tvd_out, int32_t* near_count, void* stream);
+
+/* ---- (d) path selection ------------------------------------------------------------------------ */
+/* Algorithm 2 keeps, level by level, the first accepted candidate (CASCADE_SELECT_FIRST_ACCEPT);
+ * CASCADE_SELECT_LONGEST returns the deepest node all of whose ancestors are accepted.
+ *   accept [B,T] uint8; tvd_out [B,T] float or NULL
+ *   path_nodes [B, depth+1] int32: root..end node, unused entries -1  (depth = cascade_tree_depth)
+ *   path_len [B] int32: number of accepted draft tokens (alpha of Algorithm 2)
+ *   tvd_used [B] float or NULL: the running total where the walk stops (needs tvd_out). */
+int cascade_select_path(cascade_ctx* ctx, const cascade_tree* tree, const uint8_t* accept,
+                        const float* tvd_out, int32_t mode, int32_t* path_nodes, int32_t* path_len,
+                        float* tvd_used, void* stream);
+
+/* ---- the whole step ---------------------------------------------------------------------------- */
+
+/* One pre-norm decoder layer (the workload's architecture; the paper treats the target as given):
+ * a = RMSNorm(x, gamma_attn); q,k,v = a Wq^T, a Wk^T, a Wv^T; rotary (half-split pairing) at position
+ * prefix_len[r] + depth[j]; tree attention; x += attn Wo^T; m = RMSNorm(x, gamma_mlp);
+ * x += (silu(m Wg^T) * (m Wu^T)) Wd^T.  Matrices are [out_features, in_features] elem. */
+typedef struct {
+  const float* gamma_attn; /* [h] */
+  const void* wq;          /* [Hq*D, h]  */
+  const void* wk;          /* [Hkv*D, h] */
+  const void* wv;          /* [Hkv*D, h] */
+  const void* wo;          /* [h, Hq*D]  */
+  const float* gamma_mlp;  /* [h] */
+  const void* w_gate;      /* [ffn, h] */
+  const void* w_up;        /* [ffn, h] */
+  const void* w_down;      /* [h, ffn] */
+  const void* k_prefix;    /* [R, prefix_cap, Hkv, D] this layer's cache */
+  const void* v_prefix;
+} cascade_layer;
+
+/* All arguments of one verification step.  Pointers are device pointers except `layers`, a HOST
+ * array of n_layers structs (whose members are device pointers). */
+typedef struct {
+  /* model */
+  int32_t n_layers;            /* >= 0.  0: skip the decoder layers, `hidden_in` is the head's input */
+  const cascade_layer* layers; /* host array */
+  const void* embed;           /* [V,h] elem, token embedding (n_layers > 0)                         */
+  const float* gamma_final;    /* [h]                                                                */
+  const void* w_head;          /* [V,h] elem                                                         */
+  int32_t prefix_cap;
+  const int32_t* prefix_len;   /* [R]                                                                */
+  float eps, rope_base, softmax_scale, cfg_scale, temperature;
+  /* step inputs */
+  const int32_t* tok;          /* [B,T] */
+  const float* draft_p;        /* [B,T] */
+  const float* uniforms;       /* [B,T] */
+  const void* hidden_in;       /* [R,T,h] elem, used when n_layers == 0                              */
+  /* stand-alone attention inputs, used when n_layers == 0 and q != NULL: piece (a) runs on them in
+   * the same enqueue and writes attn_out */
+  const void* q;               /* [R,T,Hq,D]  */
+  const void* k_tree;          /* [R,T,Hkv,D] */
+  const void* v_tree;
+  const void* k_prefix;        /* [R,prefix_cap,Hkv,D] */
+  const void* v_prefix;
+  void* attn_out;              /* [R,T,Hq,D] elem */
+  /* rule */
+  cascade_params params;
+  int32_t select_mode;
+  /* outputs */
+  uint8_t* accept;             /* [B,T] */
+  int32_t* path_nodes;         /* [B,depth+1] */
+  int32_t* path_len;           /* [B] */
+  float* q_relaxed;            /* [B,T] or NULL */
+  float* tvd_out;              /* [B,T] or NULL */
+  float* tvd_used;             /* [B] or NULL */
+  int32_t* near_count;         /* [B] or NULL */
+  /* optional intermediates, NULL to skip the store */
+  float* logits;               /* [B,T,V] */
+  float* feat;                 /* [B,T,h] */
+  float* scores;               /* [B,num_pairs] */
+  float* row_lse;              /* [B,T] */
+  float* hidden_out;           /* [R,T,h] float: residual stream entering the final norm (n_layers>0) */
+  void* k_tree_out;            /* [n_layers,R,T,Hkv,D] elem: rotated keys / values of the tree rows, */
+  void* v_tree_out;            /*   what a caller appends to the cache for the accepted path          */
+} cascade_step;
+
+/* Runs pieces (a)-(d) (and the decoder layers, if any) as one enqueue on `stream`. */
+int cascade_verify_step(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step, void* stream);
+
+/* Same step with the per-step inputs and results in HOST memory (pinned memory makes the copies
+ * asynchronous): tok, draft_p, uniforms [B,T] are copied in, accept [B,T], path_nodes [B,depth+1] and
+ * path_len [B] are copied back, and the call returns after the stream has been synchronised.  The
+ * corresponding pointers inside `step` are ignored (the context's own staging buffers are used);
+ * everything else in `step` is read as in cascade_verify_step. */
+int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step,
+                             const int32_t* tok_host, const float* draft_p_host, const float* uniforms_host,
+                             uint8_t* accept_host, int32_t* path_nodes_host, int32_t* path_len_host,
+                             void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CASCADE_H_ */

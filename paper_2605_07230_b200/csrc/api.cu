@@ -1,0 +1,465 @@
+// Host side of the C ABI: argument validation, context and tree descriptors, and the composition of
+// the kernels into the exported calls.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "cascade_internal.h"
+
+namespace cascade_detail {
+static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+void note_cuda_error(cudaError_t e) {
+  g_last_cuda_error = e;
+  (void)cudaGetLastError();  // clear the sticky-free error so later calls start clean
+}
+}  // namespace cascade_detail
+
+using cascade_detail::align_up;
+using cascade_detail::ceil_div;
+
+namespace {
+
+struct Carver {
+  int64_t off = 0;
+  char* base = nullptr;
+  template <typename T>
+  void take(T*& p, int64_t count) {
+    off = align_up(off, 256);
+    if (base != nullptr) p = reinterpret_cast<T*>(base + off);
+    off += count * (int64_t)sizeof(T);
+  }
+};
+
+int elem_size(const cascade_shape& s) { return s.dtype == CASCADE_BF16 ? 2 : 4; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Lays out every scratch region; with base == nullptr it only measures.
+int64_t carve(cascade_ctx* c, char* base) {
+  const cascade_shape& s = c->shape;
+  const int R = 2 * s.B, T = s.T_max;
+  const int64_t BT = (int64_t)s.B * T;
+  Carver cv;
+  cv.base = base;
+  cv.take(c->dev_error, 64);
+  const int t_pad = (int)align_up(T, 64);
+  cv.take(c->attn_part_o, (int64_t)R * s.Hq * c->attn_max_splits * t_pad * s.D);
+  cv.take(c->attn_part_ml, (int64_t)R * s.Hq * c->attn_max_splits * t_pad);
+  c->head_m_pad = (int)align_up(BT, 128);
+  if (s.dtype == CASCADE_BF16) {
+    cv.take(c->head_a_hi, (int64_t)c->head_m_pad * s.h);
+    cv.take(c->head_a_lo, (int64_t)c->head_m_pad * s.h);
+    c->head_max_tiles = ceil_div(s.V, 64) + 1;
+    cv.take(c->head_part, (int64_t)c->head_max_tiles * c->head_m_pad);
+  } else {
+    cv.take(c->head_a_f32, BT * s.h);
+  }
+  cv.take(c->feat, BT * s.h);
+  cv.take(c->feat_norm, BT);
+  cv.take(c->row_lse, BT);
+  cv.take(c->cand_parent, BT);
+  cv.take(c->cand_gparent, BT);
+  c->max_pairs = T * (CASCADE_MAX_CHILDREN + 1) / 2 + T;
+  cv.take(c->scores, (int64_t)s.B * c->max_pairs);
+  cv.take(c->q_relaxed, BT);
+  cv.take(c->tvd_out, BT);
+  cv.take(c->st_tok, BT);
+  cv.take(c->st_draft_p, BT);
+  cv.take(c->st_uniforms, BT);
+  cv.take(c->st_accept, BT);
+  cv.take(c->st_path_nodes, (int64_t)s.B * (T + 1));
+  cv.take(c->st_path_len, s.B);
+  return align_up(cv.off, 256);
+}
+
+int validate_shape(const cascade_shape* s) {
+  if (s == nullptr) return CASCADE_ERR_INVALID_ARG;
+  if (s->dtype != CASCADE_F32 && s->dtype != CASCADE_BF16) return CASCADE_ERR_INVALID_ARG;
+  if (s->B < 1 || s->T_max < 1 || s->P_max < 0 || s->h < 1 || s->Hq < 1 || s->Hkv < 1 || s->D < 1 || s->V < 1 ||
+      s->ffn < 0)
+    return CASCADE_ERR_INVALID_ARG;
+  if (s->T_max > CASCADE_MAX_TREE_ROWS) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (s->D != 64 && s->D != 128) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (s->Hq % s->Hkv != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (s->h % 64 != 0 || s->V % 8 != 0 || s->ffn % 64 != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if ((int64_t)s->B * s->T_max > (1 << 20)) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  return CASCADE_OK;
+}
+
+cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+}  // namespace
+
+extern "C" {
+
+const char* cascade_strerror(int status) {
+  switch (status) {
+    case CASCADE_OK: return "ok";
+    case CASCADE_ERR_INVALID_ARG: return "invalid argument";
+    case CASCADE_ERR_BAD_TREE: return "parent[] is not a BFS-ordered tree with contiguous sibling groups";
+    case CASCADE_ERR_WORKSPACE: return "could not allocate the context's device scratch";
+    case CASCADE_ERR_UNSUPPORTED_SHAPE: return "shape not supported by the kernels";
+    case CASCADE_ERR_CUDA: return "a CUDA call failed";
+    case CASCADE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    default: return "unknown status";
+  }
+}
+
+int cascade_create(cascade_ctx** out, const cascade_shape* shape) {
+  if (out == nullptr) return CASCADE_ERR_INVALID_ARG;
+  CASCADE_TRY(validate_shape(shape));
+  cascade_ctx* c = new (std::nothrow) cascade_ctx();
+  if (c == nullptr) return CASCADE_ERR_WORKSPACE;
+  c->shape = *shape;
+  if (cudaGetDevice(&c->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
+    (void)cudaGetLastError();
+    delete c;
+    return CASCADE_ERR_CUDA;
+  }
+  // enough KV splits that (rows x kv heads x splits) covers the SMs about twice
+  const int units = 2 * shape->B * shape->Hkv;
+  c->attn_max_splits = ceil_div(2 * c->sm_count, units);
+  if (c->attn_max_splits < 1) c->attn_max_splits = 1;
+  if (c->attn_max_splits > 16) c->attn_max_splits = 16;
+  c->ws_bytes = carve(c, nullptr);
+  if (cudaMalloc(&c->ws, (size_t)c->ws_bytes) != cudaSuccess) {
+    (void)cudaGetLastError();
+    delete c;
+    return CASCADE_ERR_WORKSPACE;
+  }
+  carve(c, c->ws);
+  if (cudaMemset(c->ws, 0, (size_t)c->ws_bytes) != cudaSuccess ||
+      cudaMallocHost(&c->host_error, 64) != cudaSuccess) {
+    (void)cudaGetLastError();
+    cudaFree(c->ws);
+    delete c;
+    return CASCADE_ERR_CUDA;
+  }
+  *c->host_error = 0;
+  *out = c;
+  return CASCADE_OK;
+}
+
+int cascade_destroy(cascade_ctx* ctx) {
+  if (ctx == nullptr) return CASCADE_ERR_INVALID_ARG;
+  cudaFree(ctx->ws);
+  cudaFreeHost(ctx->host_error);
+  delete ctx;
+  return CASCADE_OK;
+}
+
+int64_t cascade_workspace_bytes(const cascade_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
+
+int cascade_last_launch_count(const cascade_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int cascade_check(cascade_ctx* ctx, void* stream) {
+  if (ctx == nullptr) return CASCADE_ERR_INVALID_ARG;
+  cudaStream_t s = as_stream(stream);
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->host_error, ctx->dev_error, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CASCADE_CUDA_TRY(cudaStreamSynchronize(s));
+  const int word = *ctx->host_error;
+  if (word != 0) {
+    CASCADE_CUDA_TRY(cudaMemsetAsync(ctx->dev_error, 0, sizeof(int), s));
+    CASCADE_CUDA_TRY(cudaStreamSynchronize(s));
+    return CASCADE_ERR_TIMEOUT;
+  }
+  return CASCADE_OK;
+}
+
+// ---- tree ---------------------------------------------------------------------------------------------
+
+int cascade_tree_create(cascade_ctx* ctx, int32_t T, const int32_t* parent, cascade_tree** out) {
+  if (ctx == nullptr || parent == nullptr || out == nullptr || T < 1) return CASCADE_ERR_INVALID_ARG;
+  if (T > ctx->shape.T_max) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (parent[0] != -1) return CASCADE_ERR_BAD_TREE;
+  cascade_tree* t = new (std::nothrow) cascade_tree();
+  if (t == nullptr) return CASCADE_ERR_WORKSPACE;
+  t->ctx = ctx;
+  t->T = T;
+  t->parent.assign(parent, parent + T);
+  t->depth.assign(T, 0);
+  t->child_begin.assign(T, 0);
+  t->child_count.assign(T, 0);
+  t->sib_base.assign(T, 0);
+  for (int j = 1; j < T; ++j) {
+    const int p = parent[j];
+    if (p < 0 || p >= j) { delete t; return CASCADE_ERR_BAD_TREE; }
+    t->depth[j] = t->depth[p] + 1;
+    if (t->depth[j] < t->depth[j - 1]) { delete t; return CASCADE_ERR_BAD_TREE; }   // BFS order
+    if (j > 1 && p < parent[j - 1]) { delete t; return CASCADE_ERR_BAD_TREE; }      // groups contiguous
+    if (t->child_count[p] == 0) t->child_begin[p] = j;
+    t->child_count[p]++;
+    if (t->child_count[p] > CASCADE_MAX_CHILDREN) { delete t; return CASCADE_ERR_UNSUPPORTED_SHAPE; }
+    t->depth_max = t->depth[j];
+  }
+  // pair list: edge (parent[j], j) at index j-1, then the sibling pairs of each parent in order
+  for (int j = 1; j < T; ++j) {
+    t->pair_a.push_back(parent[j]);
+    t->pair_b.push_back(j);
+  }
+  for (int p = 0; p < T; ++p) {
+    t->sib_base[p] = (int)t->pair_a.size();
+    const int cb = t->child_begin[p], k = t->child_count[p];
+    for (int x = 0; x < k; ++x)
+      for (int y = x + 1; y < k; ++y) {
+        t->pair_a.push_back(cb + x);
+        t->pair_b.push_back(cb + y);
+      }
+  }
+  t->n_pairs = (int)t->pair_a.size();
+  if (t->n_pairs > ctx->max_pairs) { delete t; return CASCADE_ERR_UNSUPPORTED_SHAPE; }
+  std::vector<uint64_t> anc((size_t)T * 4, 0);
+  for (int j = 0; j < T; ++j)
+    for (int i = j; i >= 0; i = parent[i]) anc[(size_t)j * 4 + (i >> 6)] |= 1ull << (i & 63);
+
+  const int64_t n_pairs_alloc = t->n_pairs > 0 ? t->n_pairs : 1;
+  Carver cv;
+  auto layout = [&](char* base) {
+    cv = Carver();
+    cv.base = base;
+    cv.take(t->d_parent, T);
+    cv.take(t->d_depth, T);
+    cv.take(t->d_child_begin, T);
+    cv.take(t->d_child_count, T);
+    cv.take(t->d_sib_base, T);
+    cv.take(t->d_pair_a, n_pairs_alloc);
+    cv.take(t->d_pair_b, n_pairs_alloc);
+    cv.take(t->d_anc, (int64_t)T * 4);
+    return align_up(cv.off, 256);
+  };
+  const int64_t bytes = layout(nullptr);
+  if (cudaMalloc(&t->dev, (size_t)bytes) != cudaSuccess) {
+    (void)cudaGetLastError();
+    delete t;
+    return CASCADE_ERR_WORKSPACE;
+  }
+  layout(t->dev);
+  bool ok = true;
+  auto up = [&](void* dst, const void* src, size_t n) {
+    if (n && cudaMemcpy(dst, src, n, cudaMemcpyHostToDevice) != cudaSuccess) ok = false;
+  };
+  up(t->d_parent, t->parent.data(), sizeof(int32_t) * T);
+  up(t->d_depth, t->depth.data(), sizeof(int32_t) * T);
+  up(t->d_child_begin, t->child_begin.data(), sizeof(int32_t) * T);
+  up(t->d_child_count, t->child_count.data(), sizeof(int32_t) * T);
+  up(t->d_sib_base, t->sib_base.data(), sizeof(int32_t) * T);
+  up(t->d_pair_a, t->pair_a.data(), sizeof(int32_t) * t->n_pairs);
+  up(t->d_pair_b, t->pair_b.data(), sizeof(int32_t) * t->n_pairs);
+  up(t->d_anc, anc.data(), sizeof(uint64_t) * anc.size());
+  if (!ok) {
+    (void)cudaGetLastError();
+    cudaFree(t->dev);
+    delete t;
+    return CASCADE_ERR_CUDA;
+  }
+  *out = t;
+  return CASCADE_OK;
+}
+
+int cascade_tree_destroy(cascade_tree* tree) {
+  if (tree == nullptr) return CASCADE_ERR_INVALID_ARG;
+  cudaFree(tree->dev);
+  delete tree;
+  return CASCADE_OK;
+}
+
+int32_t cascade_tree_rows(const cascade_tree* tree) { return tree ? tree->T : 0; }
+int32_t cascade_tree_depth(const cascade_tree* tree) { return tree ? tree->depth_max : 0; }
+int32_t cascade_tree_num_pairs(const cascade_tree* tree) { return tree ? tree->n_pairs : 0; }
+int cascade_tree_pairs(const cascade_tree* tree, int32_t* pair_a, int32_t* pair_b) {
+  if (tree == nullptr || pair_a == nullptr || pair_b == nullptr) return CASCADE_ERR_INVALID_ARG;
+  std::memcpy(pair_a, tree->pair_a.data(), sizeof(int32_t) * tree->n_pairs);
+  std::memcpy(pair_b, tree->pair_b.data(), sizeof(int32_t) * tree->n_pairs);
+  return CASCADE_OK;
+}
+
+// ---- (a) ------------------------------------------------------------------------------------------------
+
+static int tree_attn_impl(cascade_ctx* ctx, const cascade_tree* tree, const void* q, const void* k_prefix,
+                          const void* v_prefix, int32_t prefix_cap, const int32_t* prefix_len,
+                          const void* k_tree, const void* v_tree, void* out, float softmax_scale,
+                          cudaStream_t s) {
+  if (ctx == nullptr || tree == nullptr || q == nullptr || prefix_len == nullptr || k_tree == nullptr ||
+      v_tree == nullptr || out == nullptr)
+    return CASCADE_ERR_INVALID_ARG;
+  if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
+  if (prefix_cap < 0 || prefix_cap > ctx->shape.P_max) return CASCADE_ERR_INVALID_ARG;
+  if (prefix_cap > 0 && (k_prefix == nullptr || v_prefix == nullptr)) return CASCADE_ERR_INVALID_ARG;
+  if (!(softmax_scale > 0.f)) return CASCADE_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_prefix) || !aligned16(v_prefix) || !aligned16(k_tree) || !aligned16(v_tree) ||
+      !aligned16(out))
+    return CASCADE_ERR_INVALID_ARG;
+  if (ctx->shape.dtype == CASCADE_BF16)
+    return launch_tree_attn_bf16(ctx, tree, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_prefix,
+                                 (const __nv_bfloat16*)v_prefix, prefix_cap, prefix_len,
+                                 (const __nv_bfloat16*)k_tree, (const __nv_bfloat16*)v_tree, (__nv_bfloat16*)out,
+                                 softmax_scale, s);
+  return launch_tree_attn_f32(ctx, tree, (const float*)q, (const float*)k_prefix, (const float*)v_prefix,
+                              prefix_cap, prefix_len, (const float*)k_tree, (const float*)v_tree, (float*)out,
+                              softmax_scale, s);
+}
+
+int cascade_tree_attn(cascade_ctx* ctx, const cascade_tree* tree, const void* q, const void* k_prefix,
+                      const void* v_prefix, int32_t prefix_cap, const int32_t* prefix_len,
+                      const void* k_tree, const void* v_tree, void* out, float softmax_scale, void* stream) {
+  if (ctx != nullptr) ctx->launches = 0;
+  return tree_attn_impl(ctx, tree, q, k_prefix, v_prefix, prefix_cap, prefix_len, k_tree, v_tree, out,
+                        softmax_scale, as_stream(stream));
+}
+
+// ---- (b) ------------------------------------------------------------------------------------------------
+
+static int lm_head_impl(cascade_ctx* ctx, const cascade_tree* tree, const void* hidden, const float* rms_gamma,
+                        float eps, const void* w_head, float cfg_scale, float temperature, const int32_t* tok,
+                        float* logits_out, float* feat_out, float* feat_norm_out, float* row_lse_out,
+                        float* cand_parent_out, float* cand_gparent_out, cudaStream_t s) {
+  if (ctx == nullptr || tree == nullptr || hidden == nullptr || rms_gamma == nullptr || w_head == nullptr)
+    return CASCADE_ERR_INVALID_ARG;
+  if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
+  if (!(temperature > 0.f) || !(eps >= 0.f)) return CASCADE_ERR_INVALID_ARG;
+  if (tok != nullptr && (cand_parent_out == nullptr || cand_gparent_out == nullptr)) return CASCADE_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w_head) || !aligned16(logits_out) || !aligned16(feat_out))
+    return CASCADE_ERR_INVALID_ARG;
+  if (row_lse_out == nullptr) row_lse_out = ctx->row_lse;
+  CASCADE_TRY(launch_final_norm_mix(ctx, tree->T, hidden, rms_gamma, eps, cfg_scale, 1.f / temperature, feat_out,
+                                    feat_norm_out, s));
+  if (ctx->shape.dtype == CASCADE_BF16)
+    return launch_head_bf16(ctx, tree, (const __nv_bfloat16*)w_head, tok, logits_out, row_lse_out,
+                            cand_parent_out, cand_gparent_out, s);
+  if (logits_out == nullptr) return CASCADE_ERR_INVALID_ARG;  // the fp32 path always materialises logits
+  return launch_head_f32(ctx, tree, (const float*)w_head, tok, logits_out, row_lse_out, cand_parent_out,
+                         cand_gparent_out, s);
+}
+
+int cascade_lm_head_cfg(cascade_ctx* ctx, const cascade_tree* tree, const void* hidden, const float* rms_gamma,
+                        float eps, const void* w_head, float cfg_scale, float temperature, const int32_t* tok,
+                        float* logits_out, float* feat_out, float* feat_norm_out, float* row_lse_out,
+                        float* cand_parent_out, float* cand_gparent_out, void* stream) {
+  if (ctx != nullptr) ctx->launches = 0;
+  return lm_head_impl(ctx, tree, hidden, rms_gamma, eps, w_head, cfg_scale, temperature, tok, logits_out, feat_out,
+                      feat_norm_out, row_lse_out, cand_parent_out, cand_gparent_out, as_stream(stream));
+}
+
+// ---- (c) ------------------------------------------------------------------------------------------------
+
+int cascade_similarity(cascade_ctx* ctx, const cascade_tree* tree, const float* feat, int32_t feat_dim,
+                       const float* feat_norm, float* scores_out, void* stream) {
+  if (ctx == nullptr || tree == nullptr || feat == nullptr || (scores_out == nullptr && tree->n_pairs > 0))
+    return CASCADE_ERR_INVALID_ARG;
+  if (tree->ctx != ctx || feat_dim < 4 || feat_dim % 4 != 0 || !aligned16(feat)) return CASCADE_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  return launch_similarity(ctx, tree, feat, feat_dim, feat_norm, scores_out, as_stream(stream));
+}
+
+static int validate_params(const cascade_params* p) {
+  if (p == nullptr) return CASCADE_ERR_INVALID_ARG;
+  if (!(p->tvd_budget >= 0.f)) return CASCADE_ERR_INVALID_ARG;  // also rejects NaN
+  if (p->tau_pos != p->tau_pos || p->tau_seq != p->tau_seq) return CASCADE_ERR_INVALID_ARG;
+  if (p->flags & ~(CASCADE_USE_I | CASCADE_USE_C | CASCADE_CONV_DIST_SELF)) return CASCADE_ERR_INVALID_ARG;
+  return CASCADE_OK;
+}
+
+int cascade_relaxed_accept(cascade_ctx* ctx, const cascade_tree* tree, const float* scores, const float* logits,
+                           const float* row_lse, const float* cand_parent, const float* cand_gparent,
+                           const int32_t* tok, const float* draft_p, const float* uniforms,
+                           const cascade_params* params, uint8_t* accept, float* q_relaxed, float* tvd_out,
+                           int32_t* near_count, void* stream) {
+  if (ctx == nullptr || tree == nullptr || tok == nullptr || draft_p == nullptr || uniforms == nullptr ||
+      accept == nullptr)
+    return CASCADE_ERR_INVALID_ARG;
+  if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
+  if (scores == nullptr && tree->n_pairs > 0) return CASCADE_ERR_INVALID_ARG;
+  CASCADE_TRY(validate_params(params));
+  if (logits == nullptr && (row_lse == nullptr || cand_parent == nullptr || cand_gparent == nullptr))
+    return CASCADE_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  cudaStream_t s = as_stream(stream);
+  if (logits != nullptr) {
+    CASCADE_TRY(launch_row_stats_from_logits(ctx, tree, logits, tok, ctx->row_lse, ctx->cand_parent,
+                                             ctx->cand_gparent, s));
+    row_lse = ctx->row_lse;
+    cand_parent = ctx->cand_parent;
+    cand_gparent = ctx->cand_gparent;
+  }
+  return launch_accept(ctx, tree, scores, row_lse, cand_parent, cand_gparent, tok, draft_p, uniforms, params,
+                       accept, q_relaxed, tvd_out, near_count, 0, nullptr, nullptr, nullptr, s);
+}
+
+// ---- (d) ------------------------------------------------------------------------------------------------
+
+int cascade_select_path(cascade_ctx* ctx, const cascade_tree* tree, const uint8_t* accept, const float* tvd_out,
+                        int32_t mode, int32_t* path_nodes, int32_t* path_len, float* tvd_used, void* stream) {
+  if (ctx == nullptr || tree == nullptr || accept == nullptr || path_nodes == nullptr || path_len == nullptr)
+    return CASCADE_ERR_INVALID_ARG;
+  if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
+  if (mode != CASCADE_SELECT_LONGEST && mode != CASCADE_SELECT_FIRST_ACCEPT) return CASCADE_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  return launch_select_path(ctx, tree, accept, tvd_out, mode, path_nodes, path_len, tvd_used, as_stream(stream));
+}
+
+// ---- the whole step -----------------------------------------------------------------------------------------
+
+static int verify_step_impl(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, cudaStream_t s) {
+  if (ctx == nullptr || tree == nullptr || st == nullptr) return CASCADE_ERR_INVALID_ARG;
+  if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
+  if (st->tok == nullptr || st->draft_p == nullptr || st->uniforms == nullptr || st->accept == nullptr ||
+      st->path_nodes == nullptr || st->path_len == nullptr || st->gamma_final == nullptr || st->w_head == nullptr)
+    return CASCADE_ERR_INVALID_ARG;
+  CASCADE_TRY(validate_params(&st->params));
+  if (st->select_mode != CASCADE_SELECT_LONGEST && st->select_mode != CASCADE_SELECT_FIRST_ACCEPT)
+    return CASCADE_ERR_INVALID_ARG;
+  if (st->n_layers < 0) return CASCADE_ERR_INVALID_ARG;
+  if (st->n_layers > 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;  // decoder layers: not built yet
+  if (st->hidden_in == nullptr) return CASCADE_ERR_INVALID_ARG;
+  ctx->launches = 0;
+  if (st->q != nullptr)
+    CASCADE_TRY(tree_attn_impl(ctx, tree, st->q, st->k_prefix, st->v_prefix, st->prefix_cap, st->prefix_len,
+                               st->k_tree, st->v_tree, st->attn_out, st->softmax_scale, s));
+  float* feat = st->feat ? st->feat : ctx->feat;
+  float* scores = st->scores ? st->scores : ctx->scores;
+  float* row_lse = st->row_lse ? st->row_lse : ctx->row_lse;
+  CASCADE_TRY(lm_head_impl(ctx, tree, st->hidden_in, st->gamma_final, st->eps, st->w_head, st->cfg_scale,
+                           st->temperature, st->tok, st->logits, feat, ctx->feat_norm, row_lse, ctx->cand_parent,
+                           ctx->cand_gparent, s));
+  CASCADE_TRY(launch_similarity(ctx, tree, feat, ctx->shape.h, ctx->feat_norm, scores, s));
+  return launch_accept(ctx, tree, scores, row_lse, ctx->cand_parent, ctx->cand_gparent, st->tok, st->draft_p,
+                       st->uniforms, &st->params, st->accept, st->q_relaxed ? st->q_relaxed : ctx->q_relaxed,
+                       st->tvd_out ? st->tvd_out : ctx->tvd_out, st->near_count, st->select_mode, st->path_nodes,
+                       st->path_len, st->tvd_used, s);
+}
+
+int cascade_verify_step(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step, void* stream) {
+  return verify_step_impl(ctx, tree, step, as_stream(stream));
+}
+
+int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step,
+                             const int32_t* tok_host, const float* draft_p_host, const float* uniforms_host,
+                             uint8_t* accept_host, int32_t* path_nodes_host, int32_t* path_len_host,
+                             void* stream) {
+  if (ctx == nullptr || tree == nullptr || step == nullptr || tok_host == nullptr || draft_p_host == nullptr ||
+      uniforms_host == nullptr || accept_host == nullptr || path_nodes_host == nullptr || path_len_host == nullptr)
+    return CASCADE_ERR_INVALID_ARG;
+  cudaStream_t s = as_stream(stream);
+  const size_t BT = (size_t)ctx->shape.B * tree->T;
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->st_tok, tok_host, BT * 4, cudaMemcpyHostToDevice, s));
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->st_draft_p, draft_p_host, BT * 4, cudaMemcpyHostToDevice, s));
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->st_uniforms, uniforms_host, BT * 4, cudaMemcpyHostToDevice, s));
+  cascade_step st = *step;
+  st.tok = ctx->st_tok;
+  st.draft_p = ctx->st_draft_p;
+  st.uniforms = ctx->st_uniforms;
+  st.accept = ctx->st_accept;
+  st.path_nodes = ctx->st_path_nodes;
+  st.path_len = ctx->st_path_len;
+  CASCADE_TRY(verify_step_impl(ctx, tree, &st, s));
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(accept_host, ctx->st_accept, BT, cudaMemcpyDeviceToHost, s));
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(path_nodes_host, ctx->st_path_nodes,
+                                   (size_t)ctx->shape.B * (tree->depth_max + 1) * 4, cudaMemcpyDeviceToHost, s));
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(path_len_host, ctx->st_path_len, (size_t)ctx->shape.B * 4,
+                                   cudaMemcpyDeviceToHost, s));
+  CASCADE_CUDA_TRY(cudaStreamSynchronize(s));
+  return CASCADE_OK;
+}
+
+}  // extern "C"

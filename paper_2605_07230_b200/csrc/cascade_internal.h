@@ -1,0 +1,145 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "cascade.h"
+
+#define CASCADE_CUDA_TRY(expr)                 \
+  do {                                         \
+    cudaError_t _e = (expr);                   \
+    if (_e != cudaSuccess) {                   \
+      cascade_detail::note_cuda_error(_e);     \
+      return CASCADE_ERR_CUDA;                 \
+    }                                          \
+  } while (0)
+
+#define CASCADE_TRY(expr)        \
+  do {                           \
+    int _s = (expr);             \
+    if (_s != CASCADE_OK) return _s; \
+  } while (0)
+
+namespace cascade_detail {
+void note_cuda_error(cudaError_t e);
+inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+}  // namespace cascade_detail
+
+// Bits of the device error word.
+enum : int { CASCADE_DEV_ERR_WAIT = 1 };
+
+struct cascade_ctx {
+  cascade_shape shape;
+  int device = 0;
+  int sm_count = 148;
+  int launches = 0;  // kernels enqueued by the call in progress / last call
+
+  // one device allocation, carved into the regions below
+  char* ws = nullptr;
+  int64_t ws_bytes = 0;
+
+  int* dev_error = nullptr;  // device error word
+  int* host_error = nullptr;  // pinned mirror
+
+  // tree attention, split-KV partial results
+  int attn_max_splits = 1;
+  float* attn_part_o = nullptr;   // [R*Hq*splits][T_pad][D]
+  float2* attn_part_ml = nullptr;  // [R*Hq*splits][T_pad]  (row max, row sum)
+
+  // LM head
+  int head_m_pad = 0;             // B*T_max rounded up to 128
+  __nv_bfloat16* head_a_hi = nullptr;  // [head_m_pad][h]
+  __nv_bfloat16* head_a_lo = nullptr;
+  int head_max_tiles = 0;
+  float2* head_part = nullptr;    // [head_max_tiles][head_m_pad] (tile max, tile sum of exp)
+  float* head_a_f32 = nullptr;    // [B*T_max][h] mixed operand (fp32 path)
+
+  // intermediates used when the caller passes NULL
+  float* feat = nullptr;        // [B,T,h]
+  float* feat_norm = nullptr;   // [B,T]
+  float* row_lse = nullptr;     // [B,T]
+  float* cand_parent = nullptr;   // [B,T]
+  float* cand_gparent = nullptr;  // [B,T]
+  float* scores = nullptr;      // [B,max_pairs]
+  float* q_relaxed = nullptr;   // [B,T]
+  float* tvd_out = nullptr;     // [B,T]
+  int max_pairs = 0;
+
+  // decoder layer activations (allocated when ffn > 0)
+  float* x = nullptr;            // [R*T][h] residual stream, fp32
+  __nv_bfloat16* act_hi = nullptr;  // [rows_pad][max(h,ffn,Hq*D)] GEMM operand, high part
+  __nv_bfloat16* act_lo = nullptr;
+  float* act_f32 = nullptr;      // [R*T][max(h,ffn,Hq*D)] GEMM operand (fp32 path)
+  float* gemm_out = nullptr;     // [R*T][max((Hq+2Hkv)*D, 2*ffn)] fp32 GEMM result
+  void* q_rot = nullptr;         // [R,T,Hq,D] elem
+  void* k_rot = nullptr;         // [R,T,Hkv,D] elem
+  void* v_rot = nullptr;
+  void* attn_out = nullptr;      // [R,T,Hq,D] elem
+  int rows_pad = 0;
+
+  // staging for the host-buffer entry point
+  int32_t* st_tok = nullptr;
+  float* st_draft_p = nullptr;
+  float* st_uniforms = nullptr;
+  uint8_t* st_accept = nullptr;
+  int32_t* st_path_nodes = nullptr;
+  int32_t* st_path_len = nullptr;
+};
+
+struct cascade_tree {
+  cascade_ctx* ctx = nullptr;
+  int T = 0, depth_max = 0, n_pairs = 0;
+  std::vector<int32_t> parent, depth, child_begin, child_count, pair_a, pair_b, sib_base;
+  // device copies
+  char* dev = nullptr;
+  int32_t* d_parent = nullptr;
+  int32_t* d_depth = nullptr;
+  int32_t* d_child_begin = nullptr;  // first child index (children are contiguous)
+  int32_t* d_child_count = nullptr;
+  int32_t* d_sib_base = nullptr;     // index in the pair list of the first sibling pair among node's children
+  int32_t* d_pair_a = nullptr;
+  int32_t* d_pair_b = nullptr;
+  uint64_t* d_anc = nullptr;         // [T][4] ancestor-or-self bitmask
+};
+
+// ---- kernel launchers (each returns a CASCADE_* status and bumps ctx->launches) -------------------
+
+// accept.cu
+int launch_similarity(cascade_ctx* ctx, const cascade_tree* tree, const float* feat, int feat_dim,
+                      const float* feat_norm, float* scores, cudaStream_t s);
+int launch_row_stats_from_logits(cascade_ctx* ctx, const cascade_tree* tree, const float* logits,
+                                 const int32_t* tok, float* row_lse, float* cand_parent,
+                                 float* cand_gparent, cudaStream_t s);
+int launch_accept(cascade_ctx* ctx, const cascade_tree* tree, const float* scores, const float* row_lse,
+                  const float* cand_parent, const float* cand_gparent, const int32_t* tok,
+                  const float* draft_p, const float* uniforms, const cascade_params* prm, uint8_t* accept,
+                  float* q_relaxed, float* tvd_out, int32_t* near_count,
+                  // fused path selection (skipped when path_nodes == nullptr)
+                  int select_mode, int32_t* path_nodes, int32_t* path_len, float* tvd_used, cudaStream_t s);
+int launch_select_path(cascade_ctx* ctx, const cascade_tree* tree, const uint8_t* accept,
+                       const float* tvd_out, int mode, int32_t* path_nodes, int32_t* path_len,
+                       float* tvd_used, cudaStream_t s);
+
+// attn_f32.cu / attn_bf16.cu
+int launch_tree_attn_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* q, const float* kp,
+                         const float* vp, int prefix_cap, const int32_t* prefix_len, const float* kt,
+                         const float* vt, float* out, float scale, cudaStream_t s);
+int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* q,
+                          const __nv_bfloat16* kp, const __nv_bfloat16* vp, int prefix_cap,
+                          const int32_t* prefix_len, const __nv_bfloat16* kt, const __nv_bfloat16* vt,
+                          __nv_bfloat16* out, float scale, cudaStream_t s);
+
+// head.cu (norm + mix producers, fp32 head) / gemm_tc.cu (tcgen05 GEMM)
+int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const float* gamma, float eps,
+                          float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
+                          cudaStream_t s);
+int launch_head_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* w_head, const int32_t* tok,
+                    float* logits, float* row_lse, float* cand_parent, float* cand_gparent, cudaStream_t s);
+int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* w_head,
+                     const int32_t* tok, float* logits, float* row_lse, float* cand_parent,
+                     float* cand_gparent, cudaStream_t s);
