@@ -5,6 +5,7 @@
 #include <new>
 
 #include "cascade_internal.h"
+#include "tmap.h"
 
 namespace cascade_detail {
 static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
@@ -42,6 +43,7 @@ int64_t carve(cascade_ctx* c, char* base) {
   Carver cv;
   cv.base = base;
   cv.take(c->dev_error, 64);
+  cv.take(c->gemm_counter, 64);
   const int t_pad = (int)align_up(T, 64);
   cv.take(c->attn_part_o, (int64_t)R * s.Hq * c->attn_max_splits * t_pad * s.D);
   cv.take(c->attn_part_ml, (int64_t)R * s.Hq * c->attn_max_splits * t_pad);
@@ -145,6 +147,7 @@ int cascade_destroy(cascade_ctx* ctx) {
   if (ctx == nullptr) return CASCADE_ERR_INVALID_ARG;
   cudaFree(ctx->ws);
   cudaFreeHost(ctx->host_error);
+  free_tmap_cache(ctx);
   delete ctx;
   return CASCADE_OK;
 }

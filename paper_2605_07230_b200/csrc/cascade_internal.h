@@ -45,6 +45,8 @@ struct cascade_ctx {
 
   int* dev_error = nullptr;  // device error word
   int* host_error = nullptr;  // pinned mirror
+  void* tmap_cache = nullptr; // TMA tensor maps built so far (tmap.cu)
+  unsigned int* gemm_counter = nullptr;  // CTAs-finished counter of the tensor-core GEMM
 
   // tree attention, split-KV partial results
   int attn_max_splits = 1;

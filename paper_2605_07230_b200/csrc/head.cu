@@ -5,6 +5,7 @@
 // bf16 high part plus a bf16 remainder (a = hi + lo to ~16 mantissa bits); the tensor-core GEMM adds
 // both products into one fp32 accumulator.
 #include "cascade_internal.h"
+#include "gemm_tc.h"
 
 namespace {
 
@@ -78,7 +79,63 @@ __global__ void __launch_bounds__(256) k_head_f32(const float* __restrict__ a, c
   }
 }
 
+// Logits the acceptance rule reads, straight from the operands: for draft node j the logit of tok[j]
+// under its parent's row and under its grandparent's row (Algorithm 2: q_x = gtp[x]; Eq. 3 sums).
+// One CTA per (node, prompt); 128 threads split the dot products over h.
+__global__ void __launch_bounds__(128) k_cand_logits(const __nv_bfloat16* __restrict__ a_hi,
+                                                     const __nv_bfloat16* __restrict__ a_lo,
+                                                     const __nv_bfloat16* __restrict__ W, int T, int h, int V,
+                                                     const int32_t* __restrict__ tok,
+                                                     const int32_t* __restrict__ parent,
+                                                     float* __restrict__ cand_parent,
+                                                     float* __restrict__ cand_gparent) {
+  const int j = blockIdx.x, b = blockIdx.y;
+  const size_t idx = (size_t)b * T + j;
+  __shared__ float red[2][4];
+  float dp = 0.f, dg = 0.f;
+  const int pi = parent[j];
+  const int gp = pi >= 0 ? parent[pi] : -1;
+  if (pi >= 0) {
+    const int t = tok[idx];
+    const __nv_bfloat16* w = W + (size_t)t * h;
+    const size_t rp = ((size_t)b * T + pi) * h, rg = ((size_t)b * T + (gp >= 0 ? gp : pi)) * h;
+    for (int i = threadIdx.x; i < h; i += 128) {
+      const float wv = __bfloat162float(w[i]);
+      dp += wv * (__bfloat162float(a_hi[rp + i]) + __bfloat162float(a_lo[rp + i]));
+      dg += wv * (__bfloat162float(a_hi[rg + i]) + __bfloat162float(a_lo[rg + i]));
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    dp += __shfl_xor_sync(0xffffffffu, dp, o);
+    dg += __shfl_xor_sync(0xffffffffu, dg, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    red[0][threadIdx.x >> 5] = dp;
+    red[1][threadIdx.x >> 5] = dg;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    cand_parent[idx] = pi >= 0 ? red[0][0] + red[0][1] + red[0][2] + red[0][3] : 0.f;
+    cand_gparent[idx] = gp >= 0 ? red[1][0] + red[1][1] + red[1][2] + red[1][3] : 0.f;
+  }
+}
+
 }  // namespace
+
+int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* w_head, const int32_t* tok,
+                     float* logits, float* row_lse, float* cand_parent, float* cand_gparent, cudaStream_t s) {
+  const cascade_shape& sh = ctx->shape;
+  const int M = sh.B * tree->T;
+  if (tok != nullptr) {
+    dim3 grid(tree->T, sh.B);
+    k_cand_logits<<<grid, 128, 0, s>>>(ctx->head_a_hi, ctx->head_a_lo, w_head, tree->T, sh.h, sh.V, tok,
+                                       tree->d_parent, cand_parent, cand_gparent);
+    ctx->launches++;
+    CASCADE_CUDA_TRY(cudaGetLastError());
+  }
+  return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a_hi, ctx->head_a_lo, M, logits, sh.V, ctx->head_part,
+                        cascade_detail::ceil_div(sh.V, 128), row_lse, s);
+}
 
 int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const float* gamma, float eps,
                           float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
