@@ -1,0 +1,411 @@
+// Tree-masked attention of the draft-tree rows over the prefix KV cache plus their tree ancestors
+// (Section 3 of the paper: the whole draft tree is verified by the target in one parallel pass), bf16,
+// for sm_100a.  Memory-bound decode-style kernel: every key/value row is streamed from HBM once per
+// (CFG row, head) and shared by all tree rows.
+//
+// One CTA per (KV split, query head x row block, CFG row):
+//   * a TMA producer warp streams 128-key K and V tiles (bf16, 128-byte swizzle) through a 2-stage ring;
+//   * one thread issues the tensor-core work: S = Q K^T (UMMA 128x128x128) into one of two TMEM score
+//     buffers, and O_tile = P V into one of two TMEM output buffers;
+//   * four softmax warps own the 128 TMEM lanes.  A row block holds at most 64 tree rows, and the
+//     Q tile is loaded twice (UMMA rows r and r+64 are the same tree row): lanes 0-63 take keys 0-63
+//     of every tile and lanes 64-127 take keys 64-127, so all four warps work although there are only
+//     64 rows.  Each lane keeps its own running (max, sum, output[128]) in registers (online softmax in
+//     the exp2 domain); P goes to shared memory as bf16 in the swizzled K-major layout the UMMA reads,
+//     with the other half of each row held at zero.  The two halves of a row are merged once at the end;
+//   * keys of the prefix are visible to every row up to prefix_len; keys of the tree are visible to
+//     row j iff bit i of the packed ancestor-or-self mask of j is set (one 64-bit word per lane and
+//     tile half).
+// With several KV splits each CTA writes an un-normalised partial (output, max, sum) and a second
+// small kernel merges them; with one split the CTA writes the final bf16 rows itself.
+// Every mbarrier wait is bounded (error word + normal teardown on expiry).
+#include "cascade_internal.h"
+#include "ptx.cuh"
+#include "tmap.h"
+
+namespace {
+
+constexpr int kD = 128;
+constexpr int kTileKeys = 128;
+constexpr int kRowsPerBlock = 64;
+constexpr int kThreads = 192;  // warps 0-3 softmax, warp 4 TMA, warp 5 UMMA issue + TMEM alloc
+constexpr int kQBytes = 128 * kD * 2;        // 32 KB: two 64-wide halves of [128 rows][64] bf16
+constexpr int kPBytes = 128 * kTileKeys * 2;  // 32 KB
+constexpr int kKVTileBytes = kTileKeys * kD * 2;  // 32 KB for K, same for V
+constexpr int kStageBytes = 2 * kKVTileBytes;
+constexpr int kStages = 2;
+constexpr int kSmemBytes = kQBytes + kPBytes + kStages * kStageBytes + 1024;
+constexpr int kXRow = 133;  // row stride (floats) of the half-merge exchange buffer
+
+struct AttnArgs {
+  int T, Hq, Hkv, splits, n_rb, t_pad, prefix_cap;
+  const int32_t* prefix_len;
+  const uint64_t* anc;
+  __nv_bfloat16* out;
+  float* part_o;
+  float2* part_ml;
+  float c;  // softmax_scale * log2(e)
+  int* err;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kp,
+                 const __grid_constant__ CUtensorMap tm_vp, const __grid_constant__ CUtensorMap tm_kt,
+                 const __grid_constant__ CUtensorMap tm_vt, const AttnArgs p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t q_full, kv_full[kStages], kv_empty[kStages], s_full[2], s_empty[2], p_full,
+      o_full[2], o_empty[2];
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  const uint32_t q_addr = smem_base, p_addr = smem_base + kQBytes, kv_addr = p_addr + kPBytes;
+
+  const int split = blockIdx.x, head = blockIdx.y / p.n_rb, rb = blockIdx.y % p.n_rb, r = blockIdx.z;
+  const int hk = head / (p.Hq / p.Hkv);
+  const int P = p.prefix_len[r];
+  const int n_ptiles = (P + kTileKeys - 1) / kTileKeys;
+  const int n_ttiles = (p.T + kTileKeys - 1) / kTileKeys;
+  const int total = n_ptiles + n_ttiles;
+  const int per = (total + p.splits - 1) / p.splits;
+  const int tile_begin = split * per;
+  const int tile_end = min(total, tile_begin + per);
+  const int n = max(0, tile_end - tile_begin);
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&q_full, 1);
+    for (int i = 0; i < kStages; ++i) {
+      ptx::mbar_init(&kv_full[i], 1);
+      ptx::mbar_init(&kv_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&s_full[i], 1);
+      ptx::mbar_init(&s_empty[i], 128);
+      ptx::mbar_init(&o_full[i], 1);
+      ptx::mbar_init(&o_empty[i], 128);
+    }
+    ptx::mbar_init(&p_full, 128);
+    s_abort = 0;
+    ptx::fence_mbar_init();
+  }
+  // P starts at zero: each UMMA row only ever writes its own key half
+  for (int i = threadIdx.x; i < kPBytes / 16; i += kThreads)
+    reinterpret_cast<uint4*>(smem + kQBytes)[i] = make_uint4(0, 0, 0, 0);
+  ptx::fence_proxy_async_smem();
+  if (warp == 5) {
+    ptx::tmem_alloc(&s_tmem_base, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = s_tmem_base;
+  volatile int* abort_flag = &s_abort;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
+
+  // softmax state (warps 0-3)
+  float o_acc[kD];
+  float m_run = -INFINITY, l_run = 0.f;
+
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0 && n > 0) {
+      ptx::mbar_arrive_expect_tx(&q_full, kQBytes);
+      for (int half = 0; half < 2; ++half)
+        for (int copy = 0; copy < 2; ++copy)
+          ptx::tma_load_4d(smem + half * (kQBytes / 2) + copy * (64 * 128), &tm_q, half * 64, head,
+                           rb * kRowsPerBlock, r, &q_full);
+      for (int i = 0; i < n; ++i) {
+        const int s = i % kStages;
+        const uint32_t ph = (i / kStages) & 1u;
+        if (!ptx::mbar_wait(&kv_empty[s], ph ^ 1u, abort_flag, p.err)) break;
+        const int tile = tile_begin + i;
+        const bool in_prefix = tile < n_ptiles;
+        const CUtensorMap* mk = in_prefix ? &tm_kp : &tm_kt;
+        const CUtensorMap* mv = in_prefix ? &tm_vp : &tm_vt;
+        const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys;
+        uint8_t* stage = smem + kQBytes + kPBytes + s * kStageBytes;
+        ptx::mbar_arrive_expect_tx(&kv_full[s], kStageBytes);
+        for (int half = 0; half < 2; ++half) {
+          ptx::tma_load_4d(stage + half * (kKVTileBytes / 2), mk, half * 64, hk, key0, r, &kv_full[s]);
+          ptx::tma_load_4d(stage + kKVTileBytes + half * (kKVTileBytes / 2), mv, half * 64, hk, key0, r,
+                           &kv_full[s]);
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------- UMMA issue ----------------
+    if (lane == 0 && n > 0) {
+      const uint32_t idesc_s = ptx::umma_idesc_bf16(128, kTileKeys);
+      const uint32_t idesc_o = ptx::umma_idesc_bf16_b_mn(128, kD);
+      auto issue_s = [&](int i) -> bool {
+        const int s = i % kStages;
+        if (!ptx::mbar_wait(&kv_full[s], (i / kStages) & 1u, abort_flag, p.err)) return false;
+        if (!ptx::mbar_wait(&s_empty[i & 1], ((i >> 1) & 1u) ^ 1u, abort_flag, p.err)) return false;
+        ptx::tc_fence_after();
+        const uint32_t k_addr = kv_addr + s * kStageBytes;
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
+          ptx::umma_bf16(tmem_s + (i & 1) * 128, ptx::umma_desc_sw128(q_addr + off),
+                         ptx::umma_desc_sw128(k_addr + off), idesc_s, ks != 0);
+        }
+        ptx::umma_commit(&s_full[i & 1]);
+        return true;
+      };
+      bool ok = ptx::mbar_wait(&q_full, 0, abort_flag, p.err);
+      ok = ok && issue_s(0);
+      for (int i = 0; ok && i < n; ++i) {
+        if (i + 1 < n && !issue_s(i + 1)) break;
+        if (!ptx::mbar_wait(&p_full, i & 1u, abort_flag, p.err)) break;
+        if (!ptx::mbar_wait(&o_empty[i & 1], ((i >> 1) & 1u) ^ 1u, abort_flag, p.err)) break;
+        ptx::tc_fence_after();
+        const uint32_t v_addr = kv_addr + (i % kStages) * kStageBytes + kKVTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < kTileKeys / 16; ++ks) {
+          // A = P: K-major, two 64-key column blocks of [128 rows][128 B]
+          const uint64_t pd = ptx::umma_desc_sw128(p_addr + (ks >> 2) * (128 * 128) + (ks & 3) * 32);
+          // B = V: [key][d] with d contiguous (MN-major); 16 keys = two 8-row groups of 1 KB;
+          // the two 64-wide halves of d are 16 KB apart
+          const uint64_t vd = ptx::umma_desc_sw128_strides(v_addr + ks * 2048, kKVTileBytes / 2, 1024);
+          ptx::umma_bf16(tmem_o + (i & 1) * 128, pd, vd, idesc_o, ks != 0);
+        }
+        ptx::umma_commit(&o_full[i & 1]);
+        ptx::umma_commit(&kv_empty[i % kStages]);
+      }
+    }
+  } else {
+    // ---------------- softmax warps ----------------
+    const int urow = warp * 32 + lane;        // UMMA row == TMEM lane
+    const int row_in_block = urow & 63;
+    const int khalf = urow >> 6;              // which 64 keys of each tile this lane owns
+    const int j = rb * kRowsPerBlock + row_in_block;  // tree row
+    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+#pragma unroll
+    for (int d = 0; d < kD; ++d) o_acc[d] = 0.f;
+    float alpha_prev = 1.f;
+    uint64_t anc_w[4] = {0, 0, 0, 0};
+    if (j < p.T) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) anc_w[w] = p.anc[(size_t)j * 4 + w];
+    }
+    const uint32_t p_row_addr = p_addr + khalf * (128 * 128) + urow * 128;
+    bool ok = n > 0;
+    for (int i = 0; ok && i < n; ++i) {
+      if (!ptx::mbar_wait(&s_full[i & 1], (i >> 1) & 1u, abort_flag, p.err)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const int tile = tile_begin + i;
+      const bool in_prefix = tile < n_ptiles;
+      const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys + khalf * 64;
+      // visibility of this lane's 64 keys as one 64-bit word
+      uint64_t vis;
+      if (in_prefix) {
+        const int nvis = P - key0;
+        vis = (j >= p.T || nvis <= 0) ? 0ull : (nvis >= 64 ? ~0ull : ((1ull << nvis) - 1ull));
+      } else {
+        vis = anc_w[(key0 >> 6) & 3];
+      }
+      float sc[64];
+      const uint32_t s_addr = tmem_s + lane_addr + (i & 1) * 128 + khalf * 64;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) ptx::tmem_ld16(s_addr + c * 16, sc + c * 16);
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&s_empty[i & 1]);
+      float m_new = m_run;
+#pragma unroll
+      for (int k = 0; k < 64; ++k) {
+        sc[k] = ((vis >> k) & 1ull) ? sc[k] * p.c : -INFINITY;
+        m_new = fmaxf(m_new, sc[k]);
+      }
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float alpha = m_run == -INFINITY ? 1.f : ptx::ex2(m_run - m_use);
+      float rowsum = 0.f;
+      uint32_t packed[32];
+#pragma unroll
+      for (int k = 0; k < 64; k += 2) {
+        const float p0 = ptx::ex2(sc[k] - m_use), p1 = ptx::ex2(sc[k + 1] - m_use);
+        packed[k >> 1] = ptx::pack_bf16x2(p0, p1);
+        // sum what the tensor core will actually see (bf16-rounded) so that weights add up to one
+        rowsum += __uint_as_float(packed[k >> 1] << 16) + __uint_as_float(packed[k >> 1] & 0xffff0000u);
+      }
+      if (i >= 1) {
+        // PV(i-1) complete: P may be overwritten and O_{i-1} is ready
+        if (!ptx::mbar_wait(&o_full[(i - 1) & 1], ((i - 1) >> 1) & 1u, abort_flag, p.err)) { ok = false; break; }
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        ptx::st_shared_v4(p_row_addr + ((c ^ (urow & 7)) << 4), packed[4 * c], packed[4 * c + 1], packed[4 * c + 2],
+                          packed[4 * c + 3]);
+      ptx::fence_proxy_async_smem();
+      ptx::mbar_arrive(&p_full);
+      if (i >= 1) {
+        ptx::tc_fence_after();
+        const uint32_t o_addr = tmem_o + lane_addr + ((i - 1) & 1) * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float t[16];
+          ptx::tmem_ld16(o_addr + c * 16, t);
+#pragma unroll
+          for (int k = 0; k < 16; ++k) o_acc[c * 16 + k] = o_acc[c * 16 + k] * alpha_prev + t[k];
+        }
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&o_empty[(i - 1) & 1]);
+      }
+      l_run = l_run * alpha + rowsum;
+      m_run = m_new;
+      alpha_prev = alpha;
+    }
+    if (ok && n > 0) {
+      if (ptx::mbar_wait(&o_full[(n - 1) & 1], ((n - 1) >> 1) & 1u, abort_flag, p.err)) {
+        ptx::tc_fence_after();
+        const uint32_t o_addr = tmem_o + lane_addr + ((n - 1) & 1) * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float t[16];
+          ptx::tmem_ld16(o_addr + c * 16, t);
+#pragma unroll
+          for (int k = 0; k < 16; ++k) o_acc[c * 16 + k] = o_acc[c * 16 + k] * alpha_prev + t[k];
+        }
+        ptx::tc_fence_before();
+      }
+    }
+    // ---- merge the two key halves of each row (lanes r and r+64), then write ----
+    // all UMMAs and TMA copies of this CTA have completed: the KV ring is free to reuse
+    float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);
+    ptx::named_bar_sync(1, 128);
+    if (khalf == 1) {
+      float* x = xbuf + row_in_block * kXRow;
+#pragma unroll
+      for (int d = 0; d < kD; ++d) x[d] = o_acc[d];
+      x[kD] = m_run;
+      x[kD + 1] = l_run;
+    }
+    ptx::named_bar_sync(1, 128);
+    if (khalf == 0 && j < p.T) {
+      const float* x = xbuf + row_in_block * kXRow;
+      const float m1 = x[kD], l1 = x[kD + 1];
+      const float m = fmaxf(m_run, m1);
+      const float w0 = m_run == -INFINITY ? 0.f : ptx::ex2(m_run - m);
+      const float w1 = m1 == -INFINITY ? 0.f : ptx::ex2(m1 - m);
+      const float l = l_run * w0 + l1 * w1;
+      if (p.splits == 1) {
+        const float inv = 1.f / l;
+        uint4* dst = reinterpret_cast<uint4*>(p.out + (((size_t)r * p.T + j) * p.Hq + head) * kD);
+#pragma unroll
+        for (int c = 0; c < kD / 8; ++c) {
+          uint32_t w[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int d = c * 8 + 2 * k;
+            w[k] = ptx::pack_bf16x2((o_acc[d] * w0 + x[d] * w1) * inv, (o_acc[d + 1] * w0 + x[d + 1] * w1) * inv);
+          }
+          dst[c] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      } else {
+        const size_t unit = ((size_t)r * p.Hq + head) * p.splits + split;
+        float4* dst = reinterpret_cast<float4*>(p.part_o + (unit * p.t_pad + j) * kD);
+#pragma unroll
+        for (int c = 0; c < kD / 4; ++c)
+          dst[c] = make_float4(o_acc[4 * c] * w0 + x[4 * c] * w1, o_acc[4 * c + 1] * w0 + x[4 * c + 1] * w1,
+                               o_acc[4 * c + 2] * w0 + x[4 * c + 2] * w1, o_acc[4 * c + 3] * w0 + x[4 * c + 3] * w1);
+        p.part_ml[unit * p.t_pad + j] = make_float2(m, l);
+      }
+    }
+  }
+  __syncwarp();
+  __syncthreads();
+  if (*abort_flag) __nanosleep(500000);
+  if (warp == 5) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Merge of the split-KV partials: out = sum_s w_s O_s / sum_s w_s l_s, w_s = 2^(m_s - max m).
+__global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ part_o,
+                                                      const float2* __restrict__ part_ml, int T, int Hq, int splits,
+                                                      int t_pad, __nv_bfloat16* __restrict__ out) {
+  const int j = blockIdx.x, head = blockIdx.y, r = blockIdx.z, d = threadIdx.x;
+  const size_t unit0 = ((size_t)r * Hq + head) * splits;
+  float m = -INFINITY;
+  for (int s = 0; s < splits; ++s) m = fmaxf(m, part_ml[(unit0 + s) * t_pad + j].x);
+  float acc = 0.f, l = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float2 ml = part_ml[(unit0 + s) * t_pad + j];
+    if (ml.x == -INFINITY) continue;
+    const float w = ptx::ex2(ml.x - m);
+    acc += w * part_o[((unit0 + s) * t_pad + j) * kD + d];
+    l += w * ml.y;
+  }
+  out[(((size_t)r * T + j) * Hq + head) * kD + d] = __float2bfloat16_rn(acc / l);
+}
+
+}  // namespace
+
+int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* q,
+                          const __nv_bfloat16* kp, const __nv_bfloat16* vp, int prefix_cap,
+                          const int32_t* prefix_len, const __nv_bfloat16* kt, const __nv_bfloat16* vt,
+                          __nv_bfloat16* out, float scale, cudaStream_t s) {
+  const cascade_shape& sh = ctx->shape;
+  if (sh.D != kD) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  const int T = tree->T, R = 2 * sh.B;
+  AttnArgs a;
+  a.T = T;
+  a.Hq = sh.Hq;
+  a.Hkv = sh.Hkv;
+  a.n_rb = cascade_detail::ceil_div(T, kRowsPerBlock);
+  a.t_pad = (int)cascade_detail::align_up(sh.T_max, 64);
+  a.prefix_cap = prefix_cap;
+  a.prefix_len = prefix_len;
+  a.anc = tree->d_anc;
+  a.out = out;
+  a.part_o = ctx->attn_part_o;
+  a.part_ml = ctx->attn_part_ml;
+  a.c = scale * 1.4426950408889634f;
+  a.err = ctx->dev_error;
+  // KV splits: enough CTAs to cover the SMs, never more splits than tiles, never more than the scratch holds
+  const int n_tiles = cascade_detail::ceil_div(prefix_cap, kTileKeys) + cascade_detail::ceil_div(T, kTileKeys);
+  const int units = R * sh.Hq * a.n_rb;
+  int splits = cascade_detail::ceil_div(ctx->sm_count, units);
+  if (splits > n_tiles) splits = n_tiles;
+  if (splits > ctx->attn_max_splits) splits = ctx->attn_max_splits;
+  if (splits < 1) splits = 1;
+  a.splits = splits;
+
+  const uint64_t dq[4] = {(uint64_t)kD, (uint64_t)sh.Hq, (uint64_t)T, (uint64_t)R};
+  const uint64_t sq[3] = {(uint64_t)kD, (uint64_t)sh.Hq * kD, (uint64_t)T * sh.Hq * kD};
+  const uint32_t bq[4] = {64, 1, kRowsPerBlock, 1};
+  const uint64_t dt[4] = {(uint64_t)kD, (uint64_t)sh.Hkv, (uint64_t)T, (uint64_t)R};
+  const uint64_t stt[3] = {(uint64_t)kD, (uint64_t)sh.Hkv * kD, (uint64_t)T * sh.Hkv * kD};
+  const uint32_t bkv[4] = {64, 1, kTileKeys, 1};
+  const CUtensorMap* mq = get_tmap_4d_bf16(ctx, q, dq, sq, bq);
+  const CUtensorMap* mkt = get_tmap_4d_bf16(ctx, kt, dt, stt, bkv);
+  const CUtensorMap* mvt = get_tmap_4d_bf16(ctx, vt, dt, stt, bkv);
+  const CUtensorMap* mkp = mkt;
+  const CUtensorMap* mvp = mvt;
+  if (prefix_cap > 0) {
+    const uint64_t dp[4] = {(uint64_t)kD, (uint64_t)sh.Hkv, (uint64_t)prefix_cap, (uint64_t)R};
+    const uint64_t sp[3] = {(uint64_t)kD, (uint64_t)sh.Hkv * kD, (uint64_t)prefix_cap * sh.Hkv * kD};
+    mkp = get_tmap_4d_bf16(ctx, kp, dp, sp, bkv);
+    mvp = get_tmap_4d_bf16(ctx, vp, dp, sp, bkv);
+  }
+  if (!mq || !mkt || !mvt || !mkp || !mvp) return CASCADE_ERR_CUDA;
+  static bool configured = false;
+  if (!configured) {
+    CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_tree_attn_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    configured = true;
+  }
+  dim3 grid(splits, sh.Hq * a.n_rb, R);
+  k_tree_attn_bf16<<<grid, kThreads, kSmemBytes, s>>>(*mq, *mkp, *mvp, *mkt, *mvt, a);
+  ctx->launches++;
+  CASCADE_CUDA_TRY(cudaGetLastError());
+  if (splits > 1) {
+    dim3 g2(T, sh.Hq, R);
+    k_attn_combine<<<g2, kD, 0, s>>>(ctx->attn_part_o, ctx->attn_part_ml, T, sh.Hq, splits, a.t_pad, out);
+    ctx->launches++;
+    CASCADE_CUDA_TRY(cudaGetLastError());
+  }
+  return CASCADE_OK;
+}
