@@ -109,6 +109,16 @@ int cascade_last_launch_count(const cascade_ctx* ctx);
 
 const char* cascade_strerror(int status);
 
+/* Per-kernel device timing (measurement aid, off by default).  While enabled, every kernel a call on
+ * this context enqueues is bracketed by a pair of CUDA events on the caller's stream.
+ * cascade_timing_read synchronises those events, ADDS the elapsed milliseconds and launch counts per
+ * kernel id into ms_total / launches (HOST arrays of CASCADE_KERNEL_COUNT entries, caller-zeroed) and
+ * forgets the recorded events.  cascade_kernel_name(id) names an id (NULL if out of range). */
+#define CASCADE_KERNEL_COUNT 24
+int cascade_timing_enable(cascade_ctx* ctx, int32_t on);
+int cascade_timing_read(cascade_ctx* ctx, float* ms_total, int32_t* launches);
+const char* cascade_kernel_name(int32_t id);
+
 /* The draft tree (the static tree mask of Section 3; Algorithm 2 input `tree`).
  * parent: HOST array of T entries, parent[0] = -1, 0 <= parent[j] < j, rows in BFS order (depth never
  * decreases with the index) and the children of one parent contiguous.  Builds the device-side

@@ -20,10 +20,11 @@ ERR_INVALID_ARG, ERR_BAD_TREE, ERR_WORKSPACE, ERR_UNSUPPORTED_SHAPE, ERR_CUDA, E
 F32, BF16 = 0, 1
 USE_I, USE_C, CONV_DIST_SELF = 1, 2, 4
 SELECT_LONGEST, SELECT_FIRST_ACCEPT = 0, 1
+KERNEL_COUNT = 24
 
 EXPORTS = [
     "cascade_create", "cascade_destroy", "cascade_workspace_bytes", "cascade_check", "cascade_last_launch_count",
-    "cascade_strerror", "cascade_tree_create", "cascade_tree_destroy", "cascade_tree_rows", "cascade_tree_depth",
+    "cascade_strerror", "cascade_timing_enable", "cascade_timing_read", "cascade_kernel_name", "cascade_tree_create", "cascade_tree_destroy", "cascade_tree_rows", "cascade_tree_depth",
     "cascade_tree_num_pairs", "cascade_tree_pairs", "cascade_tree_attn", "cascade_lm_head_cfg",
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
     "cascade_verify_step_host",
@@ -78,6 +79,10 @@ def lib() -> C.CDLL:
         L.cascade_workspace_bytes.argtypes = [vp]
         L.cascade_check.argtypes = [vp, vp]
         L.cascade_last_launch_count.argtypes = [vp]
+        L.cascade_timing_enable.argtypes = [vp, C.c_int32]
+        L.cascade_timing_read.argtypes = [vp, vp, vp]
+        L.cascade_kernel_name.argtypes = [C.c_int32]
+        L.cascade_kernel_name.restype = C.c_char_p
         L.cascade_tree_create.argtypes = [vp, C.c_int32, vp, C.POINTER(vp)]
         L.cascade_tree_destroy.argtypes = [vp]
         for f in ("cascade_tree_rows", "cascade_tree_depth", "cascade_tree_num_pairs"):
@@ -150,6 +155,22 @@ class Context:
 
     def check(self) -> None:
         _check(lib().cascade_check(self.handle, _stream()))
+
+    def timing_enable(self, on: bool) -> None:
+        _check(lib().cascade_timing_enable(self.handle, int(on)))
+
+    def timing_read(self) -> dict:
+        """{kernel name: (total ms, launches)} accumulated since the last read."""
+        n = KERNEL_COUNT
+        ms = (C.c_float * n)()
+        cnt = (C.c_int32 * n)()
+        _check(lib().cascade_timing_read(self.handle, ms, cnt))
+        out = {}
+        for i in range(n):
+            name = lib().cascade_kernel_name(i)
+            if name is not None and cnt[i] > 0:
+                out[name.decode()] = (float(ms[i]), int(cnt[i]))
+        return out
 
 
 class Tree:

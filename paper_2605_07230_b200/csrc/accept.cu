@@ -336,9 +336,11 @@ int launch_similarity(cascade_ctx* ctx, const cascade_tree* tree, const float* f
                       const float* feat_norm, float* scores, cudaStream_t s) {
   if (tree->n_pairs == 0) return CASCADE_OK;
   dim3 grid(tree->n_pairs, ctx->shape.B);
-  k_similarity<<<grid, 128, 0, s>>>(feat, tree->T, feat_dim, feat_norm, tree->d_pair_a, tree->d_pair_b,
-                                    tree->n_pairs, scores);
-  ctx->launches++;
+  {
+    KernelScope ks(ctx, K_SIMILARITY, s);
+    k_similarity<<<grid, 128, 0, s>>>(feat, tree->T, feat_dim, feat_norm, tree->d_pair_a, tree->d_pair_b,
+                                      tree->n_pairs, scores);
+  }
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }
@@ -347,9 +349,11 @@ int launch_row_stats_from_logits(cascade_ctx* ctx, const cascade_tree* tree, con
                                  const int32_t* tok, float* row_lse, float* cand_parent,
                                  float* cand_gparent, cudaStream_t s) {
   dim3 grid(tree->T, ctx->shape.B);
-  k_row_stats<<<grid, 256, 0, s>>>(logits, tree->T, ctx->shape.V, tok, tree->d_child_begin, tree->d_child_count,
-                                   row_lse, cand_parent, cand_gparent);
-  ctx->launches++;
+  {
+    KernelScope ks(ctx, K_ROW_STATS, s);
+    k_row_stats<<<grid, 256, 0, s>>>(logits, tree->T, ctx->shape.V, tok, tree->d_child_begin, tree->d_child_count,
+                                     row_lse, cand_parent, cand_gparent);
+  }
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }
@@ -359,12 +363,12 @@ int launch_accept(cascade_ctx* ctx, const cascade_tree* tree, const float* score
                   const float* draft_p, const float* uniforms, const cascade_params* prm, uint8_t* accept,
                   float* q_relaxed, float* tvd_out, int32_t* near_count, int select_mode, int32_t* path_nodes,
                   int32_t* path_len, float* tvd_used, cudaStream_t s) {
+  KernelScope ks(ctx, K_ACCEPT, s);
   k_accept<<<ctx->shape.B, kMaxT, 0, s>>>(tree->T, tree->depth_max, tree->n_pairs, tree->d_parent, tree->d_depth,
                                           tree->d_child_begin, tree->d_child_count, tree->d_sib_base, scores,
                                           row_lse, cand_parent, cand_gparent, tok, draft_p, uniforms, *prm, accept,
                                           q_relaxed, tvd_out, near_count, select_mode, path_nodes, path_len,
                                           tvd_used);
-  ctx->launches++;
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }
@@ -372,10 +376,10 @@ int launch_accept(cascade_ctx* ctx, const cascade_tree* tree, const float* score
 int launch_select_path(cascade_ctx* ctx, const cascade_tree* tree, const uint8_t* accept,
                        const float* tvd_out, int mode, int32_t* path_nodes, int32_t* path_len,
                        float* tvd_used, cudaStream_t s) {
+  KernelScope ks(ctx, K_SELECT_PATH, s);
   k_select_path<<<ctx->shape.B, 128, 0, s>>>(tree->T, tree->depth_max, tree->d_parent, tree->d_depth,
                                              tree->d_child_begin, tree->d_child_count, accept, tvd_out, mode,
                                              path_nodes, path_len, tvd_used);
-  ctx->launches++;
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }

@@ -107,6 +107,40 @@ const char* cascade_strerror(int status) {
   }
 }
 
+const char* cascade_kernel_name(int32_t id) {
+  static const char* names[] = {"tree_attn", "attn_combine", "tree_attn_f32", "final_norm_mix", "cand_logits",
+                                "gemm_head", "head_f32", "row_stats", "similarity", "accept", "select_path",
+                                "embed_norm", "gemm_qkv", "rope_split", "gemm_o", "resid_norm", "gemm_gate_up",
+                                "swiglu", "gemm_down", "gemm_f32", "resid_add"};
+  if (id < 0 || id >= K_KERNEL_ID_END) return nullptr;
+  return names[id];
+}
+
+int cascade_timing_enable(cascade_ctx* ctx, int32_t on) {
+  if (ctx == nullptr) return CASCADE_ERR_INVALID_ARG;
+  ctx->timing = on != 0;
+  return CASCADE_OK;
+}
+
+int cascade_timing_read(cascade_ctx* ctx, float* ms_total, int32_t* launches) {
+  if (ctx == nullptr || ms_total == nullptr || launches == nullptr) return CASCADE_ERR_INVALID_ARG;
+  int status = CASCADE_OK;
+  for (const TimedLaunch& t : ctx->timed) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(t.stop) != cudaSuccess || cudaEventElapsedTime(&ms, t.start, t.stop) != cudaSuccess) {
+      (void)cudaGetLastError();
+      status = CASCADE_ERR_CUDA;
+    } else {
+      ms_total[t.id] += ms;
+      launches[t.id] += 1;
+    }
+    ctx->event_pool.push_back(t.start);
+    ctx->event_pool.push_back(t.stop);
+  }
+  ctx->timed.clear();
+  return status;
+}
+
 int cascade_create(cascade_ctx** out, const cascade_shape* shape) {
   if (out == nullptr) return CASCADE_ERR_INVALID_ARG;
   CASCADE_TRY(validate_shape(shape));
@@ -145,6 +179,11 @@ int cascade_create(cascade_ctx** out, const cascade_shape* shape) {
 
 int cascade_destroy(cascade_ctx* ctx) {
   if (ctx == nullptr) return CASCADE_ERR_INVALID_ARG;
+  for (const TimedLaunch& t : ctx->timed) {
+    cudaEventDestroy(t.start);
+    cudaEventDestroy(t.stop);
+  }
+  for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
   cudaFree(ctx->ws);
   cudaFreeHost(ctx->host_error);
   free_tmap_cache(ctx);

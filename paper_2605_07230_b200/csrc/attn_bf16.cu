@@ -398,13 +398,15 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
     configured = true;
   }
   dim3 grid(splits, sh.Hq * a.n_rb, R);
-  k_tree_attn_bf16<<<grid, kThreads, kSmemBytes, s>>>(*mq, *mkp, *mvp, *mkt, *mvt, a);
-  ctx->launches++;
+  {
+    KernelScope ks(ctx, K_TREE_ATTN, s);
+    k_tree_attn_bf16<<<grid, kThreads, kSmemBytes, s>>>(*mq, *mkp, *mvp, *mkt, *mvt, a);
+  }
   CASCADE_CUDA_TRY(cudaGetLastError());
   if (splits > 1) {
     dim3 g2(T, sh.Hq, R);
+    KernelScope ks(ctx, K_ATTN_COMBINE, s);
     k_attn_combine<<<g2, kD, 0, s>>>(ctx->attn_part_o, ctx->attn_part_ml, T, sh.Hq, splits, a.t_pad, out);
-    ctx->launches++;
     CASCADE_CUDA_TRY(cudaGetLastError());
   }
   return CASCADE_OK;

@@ -74,9 +74,9 @@ int launch_tree_attn_f32(cascade_ctx* ctx, const cascade_tree* tree, const float
   if (smem > 48 * 1024)
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_tree_attn_f32, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(tree->T, sh.Hq, 2 * sh.B);
+  KernelScope ks(ctx, K_TREE_ATTN_F32, s);
   k_tree_attn_f32<<<grid, 128, smem, s>>>(q, kp, vp, prefix_cap, prefix_len, kt, vt, tree->d_anc, out, tree->T,
                                           sh.Hq, sh.Hkv, sh.D, scale);
-  ctx->launches++;
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }

@@ -30,6 +30,19 @@ inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 }  // namespace cascade_detail
 
+// Kernel ids for the per-kernel timing table.
+enum KernelId : int {
+  K_TREE_ATTN = 0, K_ATTN_COMBINE, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_CAND_LOGITS, K_GEMM_HEAD, K_HEAD_F32,
+  K_ROW_STATS, K_SIMILARITY, K_ACCEPT, K_SELECT_PATH, K_EMBED_NORM, K_GEMM_QKV, K_ROPE_SPLIT, K_GEMM_O,
+  K_RESID_NORM, K_GEMM_GATE_UP, K_SWIGLU, K_GEMM_DOWN, K_GEMM_F32, K_RESID_ADD, K_KERNEL_ID_END
+};
+static_assert(K_KERNEL_ID_END <= CASCADE_KERNEL_COUNT, "timing table too small");
+
+struct TimedLaunch {
+  int id;
+  cudaEvent_t start, stop;
+};
+
 // Bits of the device error word.
 enum : int { CASCADE_DEV_ERR_WAIT = 1 };
 
@@ -45,6 +58,9 @@ struct cascade_ctx {
 
   int* dev_error = nullptr;  // device error word
   int* host_error = nullptr;  // pinned mirror
+  bool timing = false;
+  std::vector<TimedLaunch> timed;        // event pairs recorded since the last read
+  std::vector<cudaEvent_t> event_pool;   // spare events
   void* tmap_cache = nullptr; // TMA tensor maps built so far (tmap.cu)
   unsigned int* gemm_counter = nullptr;  // CTAs-finished counter of the tensor-core GEMM
 
@@ -107,6 +123,33 @@ struct cascade_tree {
   int32_t* d_pair_a = nullptr;
   int32_t* d_pair_b = nullptr;
   uint64_t* d_anc = nullptr;         // [T][4] ancestor-or-self bitmask
+};
+
+// Brackets one kernel launch with events when timing is on; always counts the launch.
+struct KernelScope {
+  cascade_ctx* ctx;
+  cudaStream_t stream;
+  cudaEvent_t stop = nullptr;
+  KernelScope(cascade_ctx* c, int id, cudaStream_t s) : ctx(c), stream(s) {
+    c->launches++;
+    if (!c->timing) return;
+    cudaEvent_t ev[2];
+    for (auto& e : ev) {
+      if (!c->event_pool.empty()) {
+        e = c->event_pool.back();
+        c->event_pool.pop_back();
+      } else if (cudaEventCreate(&e) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return;
+      }
+    }
+    cudaEventRecord(ev[0], s);
+    stop = ev[1];
+    c->timed.push_back({id, ev[0], ev[1]});
+  }
+  ~KernelScope() {
+    if (stop != nullptr) cudaEventRecord(stop, stream);
+  }
 };
 
 // ---- kernel launchers (each returns a CASCADE_* status and bumps ctx->launches) -------------------

@@ -236,7 +236,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 
 int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* a_hi,
                    const __nv_bfloat16* a_lo, int M, float* C, int ldc, float2* part, int part_ld, float* lse,
-                   cudaStream_t s) {
+                   int kernel_id, cudaStream_t s) {
   if (K % kBK != 0 || M < 1 || N < 1) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   GemmArgs a;
   a.M = M;
@@ -272,8 +272,10 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   }
   const int n_tiles = a.n_ntiles * a.n_mchunks;
   const int grid = n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count;
-  k_gemm_tc<<<grid, kThreads, smem, s>>>(*tw, *thi, *tlo, a);
-  ctx->launches++;
+  {
+    KernelScope ks(ctx, kernel_id, s);
+    k_gemm_tc<<<grid, kThreads, smem, s>>>(*tw, *thi, *tlo, a);
+  }
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }

@@ -7,4 +7,4 @@
 // part[m * part_ld + tile] and row-wise log-sum-exp over n to lse[m].
 int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* a_hi,
                    const __nv_bfloat16* a_lo, int M, float* C, int ldc, float2* part, int part_ld, float* lse,
-                   cudaStream_t s);
+                   int kernel_id, cudaStream_t s);

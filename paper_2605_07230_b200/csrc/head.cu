@@ -128,13 +128,13 @@ int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bflo
   const int M = sh.B * tree->T;
   if (tok != nullptr) {
     dim3 grid(tree->T, sh.B);
+    KernelScope ks(ctx, K_CAND_LOGITS, s);
     k_cand_logits<<<grid, 128, 0, s>>>(ctx->head_a_hi, ctx->head_a_lo, w_head, tree->T, sh.h, sh.V, tok,
                                        tree->d_parent, cand_parent, cand_gparent);
-    ctx->launches++;
     CASCADE_CUDA_TRY(cudaGetLastError());
   }
   return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a_hi, ctx->head_a_lo, M, logits, sh.V, ctx->head_part,
-                        cascade_detail::ceil_div(sh.V, 128), row_lse, s);
+                        cascade_detail::ceil_div(sh.V, 128), row_lse, K_GEMM_HEAD, s);
 }
 
 int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const float* gamma, float eps,
@@ -142,6 +142,7 @@ int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const flo
                           cudaStream_t s) {
   const cascade_shape& sh = ctx->shape;
   dim3 grid(T, sh.B);
+  KernelScope ks(ctx, K_FINAL_NORM_MIX, s);
   if (sh.dtype == CASCADE_BF16)
     k_final_norm_mix<__nv_bfloat16><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(hidden), sh.B, T, sh.h,
                                                          gamma, eps, cfg_scale, inv_temperature, feat, feat_norm,
@@ -150,7 +151,6 @@ int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const flo
     k_final_norm_mix<float><<<grid, 256, 0, s>>>(static_cast<const float*>(hidden), sh.B, T, sh.h, gamma, eps,
                                                  cfg_scale, inv_temperature, feat, feat_norm, nullptr, nullptr,
                                                  ctx->head_a_f32);
-  ctx->launches++;
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }
@@ -160,8 +160,10 @@ int launch_head_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* w_h
   const cascade_shape& sh = ctx->shape;
   const int M = sh.B * tree->T;
   dim3 grid(cascade_detail::ceil_div(sh.V, 8), cascade_detail::ceil_div(M, 8));
-  k_head_f32<<<grid, 256, 0, s>>>(ctx->head_a_f32, w_head, M, sh.V, sh.h, logits);
-  ctx->launches++;
+  {
+    KernelScope ks(ctx, K_HEAD_F32, s);
+    k_head_f32<<<grid, 256, 0, s>>>(ctx->head_a_f32, w_head, M, sh.V, sh.h, logits);
+  }
   CASCADE_CUDA_TRY(cudaGetLastError());
   return launch_row_stats_from_logits(ctx, tree, logits, tok, row_lse, cand_parent, cand_gparent, s);
 }

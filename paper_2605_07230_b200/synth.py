@@ -307,6 +307,35 @@ def workload(name: str, **over) -> Workload:
     return Workload(name=name, **cfg)
 
 
+def quantize(x: np.ndarray, dtype: str) -> np.ndarray:
+    """fp32 array holding exactly the values a buffer of element type `dtype` will hold."""
+    x = np.asarray(x, np.float32)
+    return round_to_bf16(x) if dtype == "bf16" else x
+
+
+def attention_inputs(w: Workload, rng, T: int, n_kv_heads: int | None = None):
+    """Stand-alone inputs of the tree attention: q, prefix K/V, tree K/V ~ N(0,1), in the workload's type."""
+    R, H, D, P = 2 * w.B, w.n_heads, w.head_dim, w.prefix_len
+    hkv = n_kv_heads or H
+    g = lambda *shape: quantize(rng.standard_normal(shape, dtype=np.float32), w.dtype)
+    return dict(q=g(R, T, H, D), k_prefix=g(R, P, hkv, D), v_prefix=g(R, P, hkv, D), k_tree=g(R, T, hkv, D),
+                v_tree=g(R, T, hkv, D), prefix_len=np.full(R, P, np.int32))
+
+
+def tail_inputs(w: Workload, rng, parent, noise: float = 0.15):
+    """Inputs of the head / acceptance / selection pieces: a clustered codebook tied as LM head, hidden
+    states that sit near the embedding of each row's token (so a row's target mass falls on that token's
+    cluster, spread thinly over near-identical codes), stand-in drafter tokens and probabilities,
+    uniforms."""
+    T = len(parent)
+    E = quantize(clustered_codebook(rng, w.V, w.h, w.n_clusters, w.sigma), w.dtype)
+    tok, p = cluster_drafter(rng, parent, w.B, w.V, w.n_clusters)
+    base = E[np.concatenate([tok, tok], 0)]                                      # [2B,T,h]
+    hidden = quantize(base + noise * 0.02 * rng.standard_normal(base.shape, dtype=np.float32), w.dtype)
+    gamma = (1.0 + 0.1 * rng.standard_normal(w.h, dtype=np.float32)).astype(np.float32)
+    return dict(w_head=E, hidden=hidden, gamma_final=gamma, tok=tok, draft_p=p, uniforms=uniforms(rng, w.B, T))
+
+
 def uniforms(rng, B: int, T: int) -> np.ndarray:
     """Pre-drawn acceptance draws r ~ U[0,1) (the verification rule's `random()` made an input)."""
     return rng.random((B, T), dtype=np.float32)

@@ -1,0 +1,131 @@
+"""Device-resident synthetic workloads for the verification step: moves the seeded host inputs of
+`synth` into torch device buffers of the right element type and fills a `binding.Step`.
+
+Data movement and argument marshalling only; all computation happens in libcascade.so.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+from . import binding as cb
+from . import synth
+
+
+def to_device(x: np.ndarray, dtype: str, device) -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(x, np.float32))
+    if dtype == "bf16":
+        t = t.to(torch.bfloat16)
+    return t.to(device).contiguous()
+
+
+@dataclass
+class DeviceStep:
+    """One set of device buffers for a verification step plus the Step struct that points at them."""
+
+    host: dict
+    dev: dict
+    out: dict
+    step: cb.Step = field(default=None)
+
+
+class PiecesWorkload:
+    """The four hot-path pieces on stand-alone inputs (no decoder-layer glue): tree attention on
+    random q / K / V, and LM head + relaxed acceptance + path selection on hidden states that sit near
+    their tokens' embeddings.  `n_sets` independent copies of every buffer let a benchmark rotate
+    through more bytes than the L2 holds."""
+
+    def __init__(self, w: synth.Workload, device="cuda:0", n_sets: int = 1, keep_logits: bool = False,
+                 select_mode: int = cb.SELECT_LONGEST, flags: int = cb.USE_I | cb.USE_C):
+        self.w = w
+        self.device = device
+        self.parent = w.parent()
+        T = len(self.parent)
+        self.T = T
+        self.ctx = cb.Context(cb.BF16 if w.dtype == "bf16" else cb.F32, w.B, T, max(w.prefix_len, 1), w.h, w.n_heads,
+                              w.n_heads, w.head_dim, w.V, 0)
+        self.tree = cb.Tree(self.ctx, self.parent)
+        self.params = cb.Params(w.tau_pos, w.tau_seq, w.tvd_budget, flags)
+        self.sets: list[DeviceStep] = []
+        rng = np.random.default_rng(w.seed)
+        host = {}
+        host.update(synth.attention_inputs(w, rng, T))
+        host.update(synth.tail_inputs(w, rng, self.parent))
+        for s in range(n_sets):
+            if s > 0:
+                # fresh per-step inputs for every set; the big read-only tensors keep their values but
+                # live at their own addresses
+                rng_s = np.random.default_rng(w.seed * 1000 + s)
+                tok, p = synth.cluster_drafter(rng_s, self.parent, w.B, w.V, w.n_clusters)
+                base = host["w_head"][np.concatenate([tok, tok], 0)]
+                hidden = synth.quantize(base + 0.15 * 0.02 * rng_s.standard_normal(base.shape, dtype=np.float32),
+                                        w.dtype)
+                host_s = dict(host, tok=tok, draft_p=p, hidden=hidden, uniforms=synth.uniforms(rng_s, w.B, T))
+            else:
+                host_s = host
+            self.sets.append(self._make_set(host_s, keep_logits, select_mode))
+
+    def _make_set(self, host, keep_logits, select_mode) -> DeviceStep:
+        w, T, dev = self.w, self.T, self.device
+        B = w.B
+        d = {}
+        for k in ("q", "k_prefix", "v_prefix", "k_tree", "v_tree", "hidden", "w_head"):
+            d[k] = to_device(host[k], w.dtype, dev)
+        d["gamma_final"] = torch.from_numpy(host["gamma_final"]).to(dev)
+        d["prefix_len"] = torch.from_numpy(host["prefix_len"]).to(dev)
+        d["tok"] = torch.from_numpy(host["tok"]).to(dev)
+        d["draft_p"] = torch.from_numpy(host["draft_p"]).to(dev)
+        d["uniforms"] = torch.from_numpy(host["uniforms"]).to(dev)
+        el = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        o = dict(
+            attn_out=torch.zeros((2 * B, T, w.n_heads, w.head_dim), dtype=el, device=dev),
+            accept=torch.zeros((B, T), dtype=torch.uint8, device=dev),
+            path_nodes=torch.zeros((B, self.tree.depth + 1), dtype=torch.int32, device=dev),
+            path_len=torch.zeros(B, dtype=torch.int32, device=dev),
+            q_relaxed=torch.zeros((B, T), device=dev),
+            tvd_out=torch.zeros((B, T), device=dev),
+            tvd_used=torch.zeros(B, device=dev),
+            near_count=torch.zeros(B, dtype=torch.int32, device=dev),
+            feat=torch.zeros((B, T, w.h), device=dev),
+            scores=torch.zeros((B, max(self.tree.num_pairs, 1)), device=dev),
+            row_lse=torch.zeros((B, T), device=dev),
+        )
+        if keep_logits or w.dtype != "bf16":
+            o["logits"] = torch.zeros((B, T, w.V), device=dev)
+        step = cb.make_step(
+            layers=None, gamma_final=d["gamma_final"], w_head=d["w_head"], prefix_cap=w.prefix_len,
+            prefix_len=d["prefix_len"], eps=w.eps, rope_base=w.rope_base,
+            softmax_scale=float(1.0 / np.sqrt(w.head_dim)), cfg_scale=w.cfg_scale, temperature=1.0,
+            tok=d["tok"], draft_p=d["draft_p"], uniforms=d["uniforms"], hidden_in=d["hidden"],
+            q=d["q"], k_tree=d["k_tree"], v_tree=d["v_tree"],
+            k_prefix=d["k_prefix"] if w.prefix_len > 0 else None, v_prefix=d["v_prefix"] if w.prefix_len > 0 else None,
+            attn_out=o["attn_out"], params=self.params, select_mode=select_mode,
+            accept=o["accept"], path_nodes=o["path_nodes"], path_len=o["path_len"], q_relaxed=o["q_relaxed"],
+            tvd_out=o["tvd_out"], tvd_used=o["tvd_used"], near_count=o["near_count"], logits=o.get("logits"),
+            feat=o["feat"], scores=o["scores"], row_lse=o["row_lse"])
+        return DeviceStep(host=host, dev=d, out=o, step=step)
+
+    def run(self, i: int = 0) -> DeviceStep:
+        s = self.sets[i % len(self.sets)]
+        cb.cascade_verify_step(self.ctx, self.tree, s.step)
+        return s
+
+    def close(self):
+        self.tree.close()
+        self.ctx.close()
+
+    # bytes the algorithm has to move per step (each operand once), by piece
+    def algorithmic_bytes(self) -> dict:
+        w, T = self.w, self.T
+        e = 2 if w.dtype == "bf16" else 4
+        R = 2 * w.B
+        attn = R * (w.prefix_len + T) * w.n_heads * w.head_dim * 2 * e + 2 * R * T * w.n_heads * w.head_dim * e
+        head = w.V * w.h * e + R * T * w.h * e
+        return {"tree_attn": attn, "lm_head": head}
+
+    def algorithmic_flops(self) -> dict:
+        w, T = self.w, self.T
+        return {"lm_head": 2.0 * w.B * T * w.h * w.V,
+                "tree_attn": 4.0 * 2 * w.B * w.n_heads * T * (w.prefix_len + T) * w.head_dim}

@@ -13,10 +13,7 @@ from paper_2605_07230_b200 import synth
 DEV = "cuda:0"
 
 
-def quantize(x: np.ndarray, dtype: str) -> np.ndarray:
-    """fp32 array holding exactly the values the device will see."""
-    x = np.asarray(x, np.float32)
-    return synth.round_to_bf16(x) if dtype == "bf16" else x
+quantize = synth.quantize
 
 
 def to_dev(x: np.ndarray, dtype: str) -> torch.Tensor:
@@ -33,30 +30,15 @@ def make_ctx(w: synth.Workload, T: int, ffn: int = 0, P_max: int | None = None) 
                       w.n_heads, w.head_dim, w.V, ffn)
 
 
-def attention_inputs(w: synth.Workload, rng, T: int, prefix_len=None):
-    R = 2 * w.B
-    H, D, P = w.n_heads, w.head_dim, w.prefix_len
-    q = quantize(rng.standard_normal((R, T, H, D), dtype=np.float32), w.dtype)
-    kp = quantize(rng.standard_normal((R, P, H, D), dtype=np.float32), w.dtype)
-    vp = quantize(rng.standard_normal((R, P, H, D), dtype=np.float32), w.dtype)
-    kt = quantize(rng.standard_normal((R, T, H, D), dtype=np.float32), w.dtype)
-    vt = quantize(rng.standard_normal((R, T, H, D), dtype=np.float32), w.dtype)
-    plen = np.full(R, P, np.int32) if prefix_len is None else np.asarray(prefix_len, np.int32)
-    return q, kp, vp, kt, vt, plen
+def attention_inputs(w, rng, T, prefix_len=None):
+    d = synth.attention_inputs(w, rng, T)
+    plen = d["prefix_len"] if prefix_len is None else np.asarray(prefix_len, np.int32)
+    return d["q"], d["k_prefix"], d["v_prefix"], d["k_tree"], d["v_tree"], plen
 
 
-def tail_inputs(w: synth.Workload, rng, parent, noise: float = 0.15):
-    """Inputs of pieces (b)-(d): a tied clustered codebook as LM head, hidden states that sit near the
-    embedding of each row's token (so a row's target mass falls on that token's cluster), stand-in
-    drafter tokens / probabilities and uniforms."""
-    T = len(parent)
-    E = quantize(synth.clustered_codebook(rng, w.V, w.h, w.n_clusters, w.sigma), w.dtype)
-    tok, p = synth.cluster_drafter(rng, parent, w.B, w.V, w.n_clusters)
-    base = E[np.concatenate([tok, tok], 0)]                                      # [2B,T,h]
-    hidden = quantize(base + noise * 0.02 * rng.standard_normal(base.shape, dtype=np.float32), w.dtype)
-    gamma = (1.0 + 0.1 * rng.standard_normal(w.h, dtype=np.float32)).astype(np.float32)
-    u = synth.uniforms(rng, w.B, T)
-    return E, hidden, gamma, tok, p, u
+def tail_inputs(w, rng, parent, noise: float = 0.15):
+    d = synth.tail_inputs(w, rng, parent, noise)
+    return d["w_head"], d["hidden"], d["gamma_final"], d["tok"], d["draft_p"], d["uniforms"]
 
 
 def compare_decisions(parent, oracle_rows, accept_gpu, path_nodes_gpu, path_len_gpu, mode):
