@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the CASCADE tree-verification step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload janus|lumina|toy|mini] [--impl ours|reference]
+
+One "step" is one pass of the whole verification hot path over one synthetic batch.  Prints ONE JSON
+line: verify-steps/s (device-timed with CUDA events, inputs resident in HBM), the same through the
+host-buffer C-ABI entry (`e2e`), the roofline of the dominant kernel measured live with CUDA events, the
+CPU checker timed on the host cores (`cpu_baseline`), and the SM clocks seen under load.
+
+With N > 1 every rank runs an independent replica on its own GPU (the step has no exchange between
+prompts, so there is nothing to shard or reduce); the time is the max over ranks.
+`--impl reference` times the CPU checker alone (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "tree_verify_steps_per_s"
+UNIT = "steps/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed regions run."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+        self.period = period_s
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_step(w, parent, host):
+    """One whole verification step on the CPU checker (same inputs as the device step)."""
+    from oracle import cascade_oracle as O
+    scale = 1.0 / np.sqrt(w.head_dim)
+    O.tree_attention(host["q"], host["k_prefix"], host["v_prefix"], host["prefix_len"], host["k_tree"],
+                     host["v_tree"], parent, scale)
+    head, res = O.verify_tail(host["hidden"], host["gamma_final"], w.eps, host["w_head"], w.cfg_scale, 1.0,
+                              host["tok"], parent, host["draft_p"], host["uniforms"], w.tau_pos, w.tau_seq,
+                              w.tvd_budget)
+    return res
+
+
+def time_oracle(w, parent, host, budget_s=25.0, max_steps=3):
+    t0 = time.perf_counter()
+    n = 0
+    while n < max_steps and (n == 0 or (time.perf_counter() - t0) * (n + 1) / n < budget_s):
+        oracle_step(w, parent, host)
+        n += 1
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    return n / dt, n, cores
+
+
+def host_inputs(w):
+    from paper_2605_07230_b200 import synth
+    parent = w.parent()
+    rng = np.random.default_rng(w.seed)
+    host = {}
+    host.update(synth.attention_inputs(w, rng, len(parent)))
+    host.update(synth.tail_inputs(w, rng, parent))
+    return parent, host
+
+
+def run_reference(args, w):
+    """The CPU checker as the reference arm: a bounded number of whole steps on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    parent, host = host_inputs(w)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(w, parent, host)
+    steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(w, parent, host)
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    v = steps / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "tree_rows": len(parent), "prefix_len": w.prefix_len, "V": w.V,
+                   "h": w.h, "note": "CPU checker (numpy fp64), whole step; steps capped at 3"},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{steps} whole step(s) of the {w.name} workload"},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--workload", default="janus")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="enqueue every step from Python instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sets", type=int, default=0, help="rotating input sets (0 = enough to exceed the L2 per step)")
+    args = ap.parse_args()
+
+    from paper_2605_07230_b200 import synth
+    w = synth.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2605_07230_b200 import binding as cb
+    from paper_2605_07230_b200.workload import PiecesWorkload
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    dev = f"cuda:{local}"
+    peaks = load_peaks()
+
+    # enough rotating copies of the inputs that a step never finds its operands in the 126 MB L2
+    parent = w.parent()
+    T = len(parent)
+    per_set = (w.V * w.h + 2 * 2 * w.B * (w.prefix_len + T) * w.n_heads * w.head_dim) * 2
+    n_sets = args.sets or max(2, int(np.ceil(3 * 126e6 / per_set)))
+    wl = PiecesWorkload(w, device=dev, n_sets=n_sets)
+    K, W = args.steps, max(args.warmup, 3)
+
+    stream = torch.cuda.Stream()
+    graph = None
+    with torch.cuda.stream(stream):
+        for i in range(W):
+            wl.run(i)
+        stream.synchronize()
+        wl.ctx.check()
+        launches_per_step = wl.ctx.last_launch_count
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(n_sets):
+                    wl.run(i)
+            graph.replay()
+            stream.synchronize()
+
+        def run_steps(n):
+            if graph is not None:
+                for _ in range(n // n_sets):
+                    graph.replay()
+                return (n // n_sets) * n_sets
+            for i in range(n):
+                wl.run(i)
+            return n
+
+        def barrier():
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        sampler = ClockSampler(local)
+        run_steps(W)
+        barrier()
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        done = run_steps(K)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        value = world * done / (ms * 1e-3)
+
+        # per-kernel durations, measured live with CUDA events on the launching stream (no graph)
+        wl.ctx.timing_enable(True)
+        kt_steps = min(K, 300)
+        for i in range(kt_steps):
+            wl.run(i)
+        stream.synchronize()
+        timing = wl.ctx.timing_read()
+        wl.ctx.timing_enable(False)
+        clocks = sampler.stop()
+
+        # end to end through the host-buffer entry: pinned host inputs in, results out, every step
+        s0 = wl.sets[0]
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        h_tok = [pin(s.host["tok"]) for s in wl.sets]
+        h_p = [pin(s.host["draft_p"]) for s in wl.sets]
+        h_u = [pin(s.host["uniforms"]) for s in wl.sets]
+        h_acc = torch.zeros((w.B, T), dtype=torch.uint8).pin_memory()
+        h_nodes = torch.zeros((w.B, wl.tree.depth + 1), dtype=torch.int32).pin_memory()
+        h_len = torch.zeros(w.B, dtype=torch.int32).pin_memory()
+        e2e_steps = min(K, 500)
+        alpha_sum = 0
+        for i in range(3):
+            cb.cascade_verify_step_host(wl.ctx, wl.tree, wl.sets[i % n_sets].step, h_tok[i % n_sets], h_p[i % n_sets],
+                                        h_u[i % n_sets], h_acc, h_nodes, h_len)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            j = i % n_sets
+            cb.cascade_verify_step_host(wl.ctx, wl.tree, wl.sets[j].step, h_tok[j], h_p[j], h_u[j], h_acc, h_nodes,
+                                        h_len)
+            alpha_sum += int(h_len.sum())
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([e2e_s], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        wl.ctx.check()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    h2d = 3 * w.B * T * 4
+    d2h = w.B * T + w.B * (wl.tree.depth + 1) * 4 + w.B * 4
+    alg_b, alg_f = wl.algorithmic_bytes(), wl.algorithmic_flops()
+    per_kernel = {k: {"us": 1e3 * v[0] / v[1], "launches_per_step": v[1] / kt_steps} for k, v in timing.items()}
+    step_us_kernels = sum(1e3 * v[0] for v in timing.values()) / kt_steps
+    dom = max(timing, key=lambda k: timing[k][0])
+    head_us = per_kernel.get("gemm_head", {}).get("us")
+    attn_us = per_kernel.get("tree_attn", {}).get("us")
+    roofline = None
+    if head_us:
+        ach = alg_b["lm_head"] / (head_us * 1e-6) / 1e9
+        roofline = {"kernel": "gemm_head (LM head, tcgen05)", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                    "us_per_launch": head_us, "algorithmic_bytes": alg_b["lm_head"],
+                    "tensor_tflops": alg_f["lm_head"] / (head_us * 1e-6) / 1e12,
+                    "tensor_frac_of_bf16_peak": alg_f["lm_head"] / (head_us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
+    extra = {}
+    if attn_us:
+        ach = alg_b["tree_attn"] / (attn_us * 1e-6) / 1e9
+        extra["tree_attn"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": ach / peaks["hbm_gbs"], "us_per_launch": attn_us,
+                              "algorithmic_bytes": alg_b["tree_attn"]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": done, "warmup": W,
+        "ms_per_step": ms / done, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "tree_rows": T, "prefix_len": w.prefix_len, "V": w.V, "h": w.h,
+                   "heads": w.n_heads, "head_dim": w.head_dim, "cfg_scale": w.cfg_scale,
+                   "step": "tree attention + final norm + LM head/CFG + relaxed acceptance + path selection",
+                   "l2": f"inputs rotate over {n_sets} sets of {per_set / 1e6:.0f} MB (> 126 MB L2 between reuses)",
+                   "cuda_graph": graph is not None, "parallelism": "replicas" if world > 1 else "single"},
+        "accepted_tokens_per_step": alpha_sum / (e2e_steps * w.B),
+        "e2e": {"value": world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * done,
+        "launches_per_step": launches_per_step,
+        "kernels_us": {k: round(v["us"], 3) for k, v in sorted(per_kernel.items())},
+        "kernel_time_per_step_us": step_us_kernels, "dominant_kernel": dom,
+        "roofline": roofline, "roofline_other": extra,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        v, n, cores = time_oracle(w, parent, wl.sets[0].host)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{n} whole step(s) of the {w.name} workload"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
