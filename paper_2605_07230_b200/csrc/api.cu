@@ -5,6 +5,7 @@
 #include <new>
 
 #include "cascade_internal.h"
+#include "gemm_tc.h"
 #include "tmap.h"
 
 namespace cascade_detail {
@@ -43,16 +44,18 @@ int64_t carve(cascade_ctx* c, char* base) {
   Carver cv;
   cv.base = base;
   cv.take(c->dev_error, 64);
-  cv.take(c->gemm_counter, 64);
+  cv.take(c->gemm_flags, 1024);
+  cv.take(c->tail_counters, s.B);
   const int t_pad = (int)align_up(T, 64);
   cv.take(c->attn_part_o, (int64_t)R * s.Hq * c->attn_max_splits * t_pad * s.D);
   cv.take(c->attn_part_ml, (int64_t)R * s.Hq * c->attn_max_splits * t_pad);
   c->head_m_pad = (int)align_up(BT, 128);
   if (s.dtype == CASCADE_BF16) {
-    cv.take(c->head_a_hi, (int64_t)c->head_m_pad * s.h);
-    cv.take(c->head_a_lo, (int64_t)c->head_m_pad * s.h);
-    c->head_max_tiles = ceil_div(s.V, 64) + 1;
+    c->head_lo_offset = (int64_t)c->head_m_pad * s.h;
+    cv.take(c->head_a_hi, 2 * c->head_lo_offset);
+    c->head_max_tiles = ceil_div(s.V, 128);
     cv.take(c->head_part, (int64_t)c->head_max_tiles * c->head_m_pad);
+    cv.take(c->gemm_scratch, gemm_tc_scratch_floats(c->sm_count));
   } else {
     cv.take(c->head_a_f32, BT * s.h);
   }
@@ -108,10 +111,11 @@ const char* cascade_strerror(int status) {
 }
 
 const char* cascade_kernel_name(int32_t id) {
-  static const char* names[] = {"tree_attn", "attn_combine", "tree_attn_f32", "final_norm_mix", "cand_logits",
-                                "gemm_head", "head_f32", "row_stats", "similarity", "accept", "select_path",
+  static const char* names[] = {"tree_attn", "attn_combine", "tree_attn_f32", "final_norm_mix", "gemm_head",
+                                "head_f32", "row_stats", "row_lse", "similarity", "accept", "tail", "select_path",
                                 "embed_norm", "gemm_qkv", "rope_split", "gemm_o", "resid_norm", "gemm_gate_up",
                                 "swiglu", "gemm_down", "gemm_f32", "resid_add"};
+  static_assert(sizeof(names) / sizeof(names[0]) == K_KERNEL_ID_END, "one name per kernel id");
   if (id < 0 || id >= K_KERNEL_ID_END) return nullptr;
   return names[id];
 }
@@ -352,23 +356,36 @@ int cascade_tree_attn(cascade_ctx* ctx, const cascade_tree* tree, const void* q,
 
 // ---- (b) ------------------------------------------------------------------------------------------------
 
+// fold_lse: also fold the head's per-tile partials into row_lse_out here (stand-alone call); the fused
+// step leaves that to its tail kernel.
 static int lm_head_impl(cascade_ctx* ctx, const cascade_tree* tree, const void* hidden, const float* rms_gamma,
                         float eps, const void* w_head, float cfg_scale, float temperature, const int32_t* tok,
                         float* logits_out, float* feat_out, float* feat_norm_out, float* row_lse_out,
-                        float* cand_parent_out, float* cand_gparent_out, cudaStream_t s) {
+                        float* cand_parent_out, float* cand_gparent_out, bool fold_lse, cudaStream_t s) {
   if (ctx == nullptr || tree == nullptr || hidden == nullptr || rms_gamma == nullptr || w_head == nullptr)
     return CASCADE_ERR_INVALID_ARG;
   if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
   if (!(temperature > 0.f) || !(eps >= 0.f)) return CASCADE_ERR_INVALID_ARG;
   if (tok != nullptr && (cand_parent_out == nullptr || cand_gparent_out == nullptr)) return CASCADE_ERR_INVALID_ARG;
-  if (!aligned16(hidden) || !aligned16(w_head) || !aligned16(logits_out) || !aligned16(feat_out))
+  if (!aligned16(hidden) || !aligned16(w_head) || !aligned16(logits_out) || !aligned16(feat_out) ||
+      !aligned16(rms_gamma))
     return CASCADE_ERR_INVALID_ARG;
   if (row_lse_out == nullptr) row_lse_out = ctx->row_lse;
   CASCADE_TRY(launch_final_norm_mix(ctx, tree->T, hidden, rms_gamma, eps, cfg_scale, 1.f / temperature, feat_out,
-                                    feat_norm_out, s));
-  if (ctx->shape.dtype == CASCADE_BF16)
-    return launch_head_bf16(ctx, tree, (const __nv_bfloat16*)w_head, tok, logits_out, row_lse_out,
-                            cand_parent_out, cand_gparent_out, s);
+                                    feat_norm_out, tok ? cand_parent_out : nullptr, tok ? cand_gparent_out : nullptr,
+                                    s));
+  if (ctx->shape.dtype == CASCADE_BF16) {
+    CASCADE_TRY(launch_head_bf16(ctx, tree, (const __nv_bfloat16*)w_head, tok, logits_out, cand_parent_out,
+                                 cand_gparent_out, s));
+    if (!fold_lse) return CASCADE_OK;
+    TailWork w;
+    w.kernel_id = K_ROW_LSE;
+    w.part = ctx->head_part;
+    w.part_ld = ctx->head_max_tiles;
+    w.n_tiles = ceil_div(ctx->shape.V, 128);
+    w.row_lse = row_lse_out;
+    return launch_tail(ctx, tree, w, s);
+  }
   if (logits_out == nullptr) return CASCADE_ERR_INVALID_ARG;  // the fp32 path always materialises logits
   return launch_head_f32(ctx, tree, (const float*)w_head, tok, logits_out, row_lse_out, cand_parent_out,
                          cand_gparent_out, s);
@@ -380,7 +397,7 @@ int cascade_lm_head_cfg(cascade_ctx* ctx, const cascade_tree* tree, const void* 
                         float* cand_parent_out, float* cand_gparent_out, void* stream) {
   if (ctx != nullptr) ctx->launches = 0;
   return lm_head_impl(ctx, tree, hidden, rms_gamma, eps, w_head, cfg_scale, temperature, tok, logits_out, feat_out,
-                      feat_norm_out, row_lse_out, cand_parent_out, cand_gparent_out, as_stream(stream));
+                      feat_norm_out, row_lse_out, cand_parent_out, cand_gparent_out, true, as_stream(stream));
 }
 
 // ---- (c) ------------------------------------------------------------------------------------------------
@@ -391,7 +408,13 @@ int cascade_similarity(cascade_ctx* ctx, const cascade_tree* tree, const float* 
     return CASCADE_ERR_INVALID_ARG;
   if (tree->ctx != ctx || feat_dim < 4 || feat_dim % 4 != 0 || !aligned16(feat)) return CASCADE_ERR_INVALID_ARG;
   ctx->launches = 0;
-  return launch_similarity(ctx, tree, feat, feat_dim, feat_norm, scores_out, as_stream(stream));
+  TailWork w;
+  w.kernel_id = K_SIMILARITY;
+  w.feat = feat;
+  w.feat_dim = feat_dim;
+  w.feat_norm = feat_norm;
+  w.scores = scores_out;
+  return launch_tail(ctx, tree, w, as_stream(stream));
 }
 
 static int validate_params(const cascade_params* p) {
@@ -424,8 +447,21 @@ int cascade_relaxed_accept(cascade_ctx* ctx, const cascade_tree* tree, const flo
     cand_parent = ctx->cand_parent;
     cand_gparent = ctx->cand_gparent;
   }
-  return launch_accept(ctx, tree, scores, row_lse, cand_parent, cand_gparent, tok, draft_p, uniforms, params,
-                       accept, q_relaxed, tvd_out, near_count, 0, nullptr, nullptr, nullptr, s);
+  TailWork w;
+  w.kernel_id = K_ACCEPT;
+  w.scores = const_cast<float*>(scores);
+  w.row_lse = const_cast<float*>(row_lse);
+  w.prm = params;
+  w.cand_parent = cand_parent;
+  w.cand_gparent = cand_gparent;
+  w.tok = tok;
+  w.draft_p = draft_p;
+  w.uniforms = uniforms;
+  w.accept = accept;
+  w.q_relaxed = q_relaxed;
+  w.tvd_out = tvd_out;
+  w.near_count = near_count;
+  return launch_tail(ctx, tree, w, s);
 }
 
 // ---- (d) ------------------------------------------------------------------------------------------------
@@ -459,16 +495,38 @@ static int verify_step_impl(cascade_ctx* ctx, const cascade_tree* tree, const ca
     CASCADE_TRY(tree_attn_impl(ctx, tree, st->q, st->k_prefix, st->v_prefix, st->prefix_cap, st->prefix_len,
                                st->k_tree, st->v_tree, st->attn_out, st->softmax_scale, s));
   float* feat = st->feat ? st->feat : ctx->feat;
-  float* scores = st->scores ? st->scores : ctx->scores;
   float* row_lse = st->row_lse ? st->row_lse : ctx->row_lse;
+  const bool bf16 = ctx->shape.dtype == CASCADE_BF16;
   CASCADE_TRY(lm_head_impl(ctx, tree, st->hidden_in, st->gamma_final, st->eps, st->w_head, st->cfg_scale,
                            st->temperature, st->tok, st->logits, feat, ctx->feat_norm, row_lse, ctx->cand_parent,
-                           ctx->cand_gparent, s));
-  CASCADE_TRY(launch_similarity(ctx, tree, feat, ctx->shape.h, ctx->feat_norm, scores, s));
-  return launch_accept(ctx, tree, scores, row_lse, ctx->cand_parent, ctx->cand_gparent, st->tok, st->draft_p,
-                       st->uniforms, &st->params, st->accept, st->q_relaxed ? st->q_relaxed : ctx->q_relaxed,
-                       st->tvd_out ? st->tvd_out : ctx->tvd_out, st->near_count, st->select_mode, st->path_nodes,
-                       st->path_len, st->tvd_used, s);
+                           ctx->cand_gparent, false, s));
+  // cosines, row log-sum-exp (bf16: folded from the head's partials), the rule and the path: one launch
+  TailWork w;
+  w.feat = feat;
+  w.feat_dim = ctx->shape.h;
+  w.feat_norm = ctx->feat_norm;
+  w.scores = st->scores ? st->scores : ctx->scores;
+  if (bf16) {
+    w.part = ctx->head_part;
+    w.part_ld = ctx->head_max_tiles;
+    w.n_tiles = ceil_div(ctx->shape.V, 128);
+  }
+  w.row_lse = row_lse;
+  w.prm = &st->params;
+  w.cand_parent = ctx->cand_parent;
+  w.cand_gparent = ctx->cand_gparent;
+  w.tok = st->tok;
+  w.draft_p = st->draft_p;
+  w.uniforms = st->uniforms;
+  w.accept = st->accept;
+  w.q_relaxed = st->q_relaxed ? st->q_relaxed : ctx->q_relaxed;
+  w.tvd_out = st->tvd_out ? st->tvd_out : ctx->tvd_out;
+  w.near_count = st->near_count;
+  w.select_mode = st->select_mode;
+  w.path_nodes = st->path_nodes;
+  w.path_len = st->path_len;
+  w.tvd_used = st->tvd_used;
+  return launch_tail(ctx, tree, w, s);
 }
 
 int cascade_verify_step(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step, void* stream) {

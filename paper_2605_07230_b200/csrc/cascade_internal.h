@@ -32,8 +32,8 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // Kernel ids for the per-kernel timing table.
 enum KernelId : int {
-  K_TREE_ATTN = 0, K_ATTN_COMBINE, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_CAND_LOGITS, K_GEMM_HEAD, K_HEAD_F32,
-  K_ROW_STATS, K_SIMILARITY, K_ACCEPT, K_SELECT_PATH, K_EMBED_NORM, K_GEMM_QKV, K_ROPE_SPLIT, K_GEMM_O,
+  K_TREE_ATTN = 0, K_ATTN_COMBINE, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_GEMM_HEAD, K_HEAD_F32, K_ROW_STATS,
+  K_ROW_LSE, K_SIMILARITY, K_ACCEPT, K_TAIL, K_SELECT_PATH, K_EMBED_NORM, K_GEMM_QKV, K_ROPE_SPLIT, K_GEMM_O,
   K_RESID_NORM, K_GEMM_GATE_UP, K_SWIGLU, K_GEMM_DOWN, K_GEMM_F32, K_RESID_ADD, K_KERNEL_ID_END
 };
 static_assert(K_KERNEL_ID_END <= CASCADE_KERNEL_COUNT, "timing table too small");
@@ -62,7 +62,8 @@ struct cascade_ctx {
   std::vector<TimedLaunch> timed;        // event pairs recorded since the last read
   std::vector<cudaEvent_t> event_pool;   // spare events
   void* tmap_cache = nullptr; // TMA tensor maps built so far (tmap.cu)
-  unsigned int* gemm_counter = nullptr;  // CTAs-finished counter of the tensor-core GEMM
+  float* gemm_scratch = nullptr;         // tensor-core GEMM: partial accumulators of tiles split between CTAs
+  unsigned int* gemm_flags = nullptr;    // one hand-off flag per CTA (zero between launches)
 
   // tree attention, split-KV partial results
   int attn_max_splits = 1;
@@ -71,11 +72,12 @@ struct cascade_ctx {
 
   // LM head
   int head_m_pad = 0;             // B*T_max rounded up to 128
-  __nv_bfloat16* head_a_hi = nullptr;  // [head_m_pad][h]
-  __nv_bfloat16* head_a_lo = nullptr;
+  __nv_bfloat16* head_a_hi = nullptr;  // [head_m_pad][h], followed by the remainder part [head_m_pad][h]
+  int64_t head_lo_offset = 0;          // elements from head_a_hi to the remainder part
   int head_max_tiles = 0;
   float2* head_part = nullptr;    // [head_max_tiles][head_m_pad] (tile max, tile sum of exp)
   float* head_a_f32 = nullptr;    // [B*T_max][h] mixed operand (fp32 path)
+  unsigned int* tail_counters = nullptr;  // [B] CTAs-finished counters of the tail kernel (zero between launches)
 
   // intermediates used when the caller passes NULL
   float* feat = nullptr;        // [B,T,h]
@@ -155,17 +157,38 @@ struct KernelScope {
 // ---- kernel launchers (each returns a CASCADE_* status and bumps ctx->launches) -------------------
 
 // accept.cu
-int launch_similarity(cascade_ctx* ctx, const cascade_tree* tree, const float* feat, int feat_dim,
-                      const float* feat_norm, float* scores, cudaStream_t s);
+// One launch of the tail kernel: any of (cosines, row log-sum-exp from the head's partials, the rule).
+struct TailWork {
+  int kernel_id = K_TAIL;
+  // cosines of the tree's pair list (skipped when feat == nullptr); written to `scores`
+  const float* feat = nullptr;
+  int feat_dim = 0;
+  const float* feat_norm = nullptr;
+  float* scores = nullptr;      // [B, n_pairs]: output of the cosines, input of the rule
+  // row log-sum-exp from per-tile partials (skipped when part == nullptr); written to `row_lse`
+  const float2* part = nullptr;
+  int part_ld = 0, n_tiles = 0;
+  float* row_lse = nullptr;     // [B, T]: output of the fold, input of the rule
+  // the rule (skipped when prm == nullptr) and path selection (skipped when path_nodes == nullptr)
+  const cascade_params* prm = nullptr;
+  const float* cand_parent = nullptr;
+  const float* cand_gparent = nullptr;
+  const int32_t* tok = nullptr;
+  const float* draft_p = nullptr;
+  const float* uniforms = nullptr;
+  uint8_t* accept = nullptr;
+  float* q_relaxed = nullptr;
+  float* tvd_out = nullptr;
+  int32_t* near_count = nullptr;
+  int select_mode = 0;
+  int32_t* path_nodes = nullptr;
+  int32_t* path_len = nullptr;
+  float* tvd_used = nullptr;
+};
+int launch_tail(cascade_ctx* ctx, const cascade_tree* tree, const TailWork& w, cudaStream_t s);
 int launch_row_stats_from_logits(cascade_ctx* ctx, const cascade_tree* tree, const float* logits,
                                  const int32_t* tok, float* row_lse, float* cand_parent,
                                  float* cand_gparent, cudaStream_t s);
-int launch_accept(cascade_ctx* ctx, const cascade_tree* tree, const float* scores, const float* row_lse,
-                  const float* cand_parent, const float* cand_gparent, const int32_t* tok,
-                  const float* draft_p, const float* uniforms, const cascade_params* prm, uint8_t* accept,
-                  float* q_relaxed, float* tvd_out, int32_t* near_count,
-                  // fused path selection (skipped when path_nodes == nullptr)
-                  int select_mode, int32_t* path_nodes, int32_t* path_len, float* tvd_used, cudaStream_t s);
 int launch_select_path(cascade_ctx* ctx, const cascade_tree* tree, const uint8_t* accept,
                        const float* tvd_out, int mode, int32_t* path_nodes, int32_t* path_len,
                        float* tvd_used, cudaStream_t s);
@@ -180,11 +203,13 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
                           __nv_bfloat16* out, float scale, cudaStream_t s);
 
 // head.cu (norm + mix producers, fp32 head) / gemm_tc.cu (tcgen05 GEMM)
+// cand_parent / cand_gparent (may be null) are cleared here; the head fills the entries that exist.
 int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const float* gamma, float eps,
                           float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
-                          cudaStream_t s);
+                          float* cand_parent, float* cand_gparent, cudaStream_t s);
 int launch_head_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* w_head, const int32_t* tok,
                     float* logits, float* row_lse, float* cand_parent, float* cand_gparent, cudaStream_t s);
+// bf16 head: logits (optional), per-tile softmax partials into the context, gathered candidate logits.
+// The row log-sum-exp is folded from the partials by launch_tail.
 int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* w_head,
-                     const int32_t* tok, float* logits, float* row_lse, float* cand_parent,
-                     float* cand_gparent, cudaStream_t s);
+                     const int32_t* tok, float* logits, float* cand_parent, float* cand_gparent, cudaStream_t s);

@@ -1,10 +1,26 @@
 #pragma once
 #include "cascade_internal.h"
 
+// What the tensor-core GEMM does with a finished tile (all members optional).
+struct GemmEpilogue {
+  float* C = nullptr;      // [M][ldc] fp32 result
+  int ldc = 0;
+  int accumulate = 0;      // 1: C += result (residual add), 0: C = result
+  float2* part = nullptr;  // per-(row, 128-wide tile) softmax partials (max, sum of exp): part[m * part_ld + tile]
+  int part_ld = 0;
+  // gather of the logits the acceptance rule reads (needs part): for idx = b * T + j,
+  // cand_parent[idx] = C[b * T + parent[j]][tok[idx]], cand_gparent[idx] likewise for the grandparent
+  const int32_t* tok = nullptr;
+  const int32_t* parent = nullptr;
+  int T = 0, n_rows = 0;
+  float* cand_parent = nullptr;
+  float* cand_gparent = nullptr;
+};
+
 // C[m][n] = sum_k (a_hi[m][k] + a_lo[m][k]) * W[n][k] on the tensor cores (see gemm_tc.cu).
-// W [N][K] bf16, a_hi/a_lo [M][K] bf16, K a multiple of 64.  C (fp32, row stride ldc) may be null.
-// With part != null the kernel also writes per-(row, 128-wide tile) softmax partials to
-// part[m * part_ld + tile] and row-wise log-sum-exp over n to lse[m].
+// W [N][K] bf16; a_hi [M][K] bf16 and the remainder a_lo = a_hi + lo_offset elements (same layout);
+// K a multiple of 8.  Uses the context's split-tile scratch: calls on one context must not overlap.
 int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* a_hi,
-                   const __nv_bfloat16* a_lo, int M, float* C, int ldc, float2* part, int part_ld, float* lse,
-                   int kernel_id, cudaStream_t s);
+                   int64_t lo_offset, int M, const GemmEpilogue& epi, int kernel_id, cudaStream_t s);
+// Floats of scratch the split-tile hand-off needs for a device with `sm_count` SMs.
+int64_t gemm_tc_scratch_floats(int sm_count);

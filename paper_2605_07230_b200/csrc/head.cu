@@ -9,58 +9,130 @@
 
 namespace {
 
-__device__ __forceinline__ float load_elem(const float* p, size_t i) { return p[i]; }
-__device__ __forceinline__ float load_elem(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
+// 8 consecutive elements of a row as floats (16-byte loads for bf16, 2 x 16 bytes for fp32)
+__device__ __forceinline__ void load8(const float* p, float* v) {
+  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float* v) {
+  const uint4 r = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
 
-__device__ __forceinline__ float block_sum_256(float v, float* red) {
+constexpr int kNormThreads = 256;
+constexpr int kNormChunks = 4;  // rows of up to 256 * 8 * 4 = 8192 elements stay in registers
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   __syncthreads();
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
   __syncthreads();
   float t = 0.f;
-  for (int i = 0; i < 8; ++i) t += red[i];
+  for (int i = 0; i < kNormThreads / 32; ++i) t += red[i];
   return t;
 }
 
+// One CTA per (tree row, prompt): RMSNorm of the cond and uncond rows, features, guidance mix.
+// h is a multiple of 8.  Rows longer than the register budget are read a second time.
 template <typename E>
-__global__ void __launch_bounds__(256) k_final_norm_mix(const E* __restrict__ hidden, int B, int T, int h,
-                                                        const float* __restrict__ gamma, float eps, float s,
-                                                        float inv_temp, float* __restrict__ feat,
-                                                        float* __restrict__ feat_norm,
-                                                        __nv_bfloat16* __restrict__ a_hi,
-                                                        __nv_bfloat16* __restrict__ a_lo,
-                                                        float* __restrict__ a_f32) {
-  __shared__ float red[8];
+__global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __restrict__ hidden, int B, int T, int h,
+                                                                 const float* __restrict__ gamma, float eps, float s,
+                                                                 float inv_temp, float* __restrict__ feat,
+                                                                 float* __restrict__ feat_norm,
+                                                                 __nv_bfloat16* __restrict__ a_hi,
+                                                                 __nv_bfloat16* __restrict__ a_lo,
+                                                                 float* __restrict__ a_f32,
+                                                                 float* __restrict__ cand_parent,
+                                                                 float* __restrict__ cand_gparent) {
+  __shared__ float red[kNormThreads / 32];
   const int j = blockIdx.x, b = blockIdx.y;
-  const size_t row_c = ((size_t)b * T + j) * h, row_u = ((size_t)(B + b) * T + j) * h;
-  float ss_c = 0.f, ss_u = 0.f;
-  for (int i = threadIdx.x; i < h; i += 256) {
-    const float c = load_elem(hidden, row_c + i), u = load_elem(hidden, row_u + i);
-    ss_c += c * c;
-    ss_u += u * u;
-  }
-  ss_c = block_sum_256(ss_c, red);
-  ss_u = block_sum_256(ss_u, red);
-  const float rc = rsqrtf(ss_c / h + eps), ru = rsqrtf(ss_u / h + eps);
-  float nn = 0.f;
   const size_t m = (size_t)b * T + j;
-  for (int i = threadIdx.x; i < h; i += 256) {
-    const float g = gamma[i];
-    const float nc = load_elem(hidden, row_c + i) * rc * g;
-    const float nu = load_elem(hidden, row_u + i) * ru * g;
-    nn += nc * nc;
-    if (feat != nullptr) feat[m * h + i] = nc;
-    const float a = (nu + s * (nc - nu)) * inv_temp;
-    if (a_hi != nullptr) {
-      const __nv_bfloat16 hi = __float2bfloat16_rn(a);
-      a_hi[m * h + i] = hi;
-      a_lo[m * h + i] = __float2bfloat16_rn(a - __bfloat162float(hi));
-    } else {
-      a_f32[m * h + i] = a;
+  const E* row_c = hidden + m * h;
+  const E* row_u = hidden + ((size_t)(B + b) * T + j) * h;
+  const int n8 = h / 8;
+  float c[kNormChunks][8], u[kNormChunks][8];
+  float ss_c = 0.f, ss_u = 0.f;
+#pragma unroll
+  for (int k = 0; k < kNormChunks; ++k) {
+    const int i = threadIdx.x + k * kNormThreads;
+    if (i < n8) {
+      load8(row_c + 8 * i, c[k]);
+      load8(row_u + 8 * i, u[k]);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        ss_c += c[k][e] * c[k][e];
+        ss_u += u[k][e] * u[k][e];
+      }
     }
   }
-  nn = block_sum_256(nn, red);
-  if (threadIdx.x == 0 && feat_norm != nullptr) feat_norm[m] = sqrtf(nn);
+  for (int i = threadIdx.x + kNormChunks * kNormThreads; i < n8; i += kNormThreads) {
+    float tc[8], tu[8];
+    load8(row_c + 8 * i, tc);
+    load8(row_u + 8 * i, tu);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      ss_c += tc[e] * tc[e];
+      ss_u += tu[e] * tu[e];
+    }
+  }
+  ss_c = block_sum(ss_c, red);
+  ss_u = block_sum(ss_u, red);
+  const float rc = rsqrtf(ss_c / h + eps), ru = rsqrtf(ss_u / h + eps);
+  float nn = 0.f;
+  auto emit = [&](int i, const float* vc, const float* vu) {
+    float g[8], nc[8], a[8];
+    load8(gamma + 8 * i, g);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      nc[e] = vc[e] * rc * g[e];
+      const float nu = vu[e] * ru * g[e];
+      nn += nc[e] * nc[e];
+      a[e] = (nu + s * (nc[e] - nu)) * inv_temp;
+    }
+    const size_t o = m * h + 8 * (size_t)i;
+    if (feat != nullptr) {
+      *reinterpret_cast<float4*>(feat + o) = make_float4(nc[0], nc[1], nc[2], nc[3]);
+      *reinterpret_cast<float4*>(feat + o + 4) = make_float4(nc[4], nc[5], nc[6], nc[7]);
+    }
+    if (a_hi != nullptr) {
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(a[2 * e]), h1 = __float2bfloat16_rn(a[2 * e + 1]);
+        const __nv_bfloat16 l0 = __float2bfloat16_rn(a[2 * e] - __bfloat162float(h0));
+        const __nv_bfloat16 l1 = __float2bfloat16_rn(a[2 * e + 1] - __bfloat162float(h1));
+        hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      }
+      *reinterpret_cast<uint4*>(a_hi + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(a_lo + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    } else {
+      *reinterpret_cast<float4*>(a_f32 + o) = make_float4(a[0], a[1], a[2], a[3]);
+      *reinterpret_cast<float4*>(a_f32 + o + 4) = make_float4(a[4], a[5], a[6], a[7]);
+    }
+  };
+#pragma unroll
+  for (int k = 0; k < kNormChunks; ++k) {
+    const int i = threadIdx.x + k * kNormThreads;
+    if (i < n8) emit(i, c[k], u[k]);
+  }
+  for (int i = threadIdx.x + kNormChunks * kNormThreads; i < n8; i += kNormThreads) {
+    float tc[8], tu[8];
+    load8(row_c + 8 * i, tc);
+    load8(row_u + 8 * i, tu);
+    emit(i, tc, tu);
+  }
+  nn = block_sum(nn, red);
+  if (threadIdx.x == 0) {
+    if (feat_norm != nullptr) feat_norm[m] = sqrtf(nn);
+    if (cand_parent != nullptr) cand_parent[m] = 0.f;
+    if (cand_gparent != nullptr) cand_gparent[m] = 0.f;
+  }
 }
 
 // logits[m][v] = sum_k a[m][k] W[v][k]; a warp per vocabulary row, 8 operand rows per CTA.
@@ -79,78 +151,42 @@ __global__ void __launch_bounds__(256) k_head_f32(const float* __restrict__ a, c
   }
 }
 
-// Logits the acceptance rule reads, straight from the operands: for draft node j the logit of tok[j]
-// under its parent's row and under its grandparent's row (Algorithm 2: q_x = gtp[x]; Eq. 3 sums).
-// One CTA per (node, prompt); 128 threads split the dot products over h.
-__global__ void __launch_bounds__(128) k_cand_logits(const __nv_bfloat16* __restrict__ a_hi,
-                                                     const __nv_bfloat16* __restrict__ a_lo,
-                                                     const __nv_bfloat16* __restrict__ W, int T, int h, int V,
-                                                     const int32_t* __restrict__ tok,
-                                                     const int32_t* __restrict__ parent,
-                                                     float* __restrict__ cand_parent,
-                                                     float* __restrict__ cand_gparent) {
-  const int j = blockIdx.x, b = blockIdx.y;
-  const size_t idx = (size_t)b * T + j;
-  __shared__ float red[2][4];
-  float dp = 0.f, dg = 0.f;
-  const int pi = parent[j];
-  const int gp = pi >= 0 ? parent[pi] : -1;
-  if (pi >= 0) {
-    const int t = tok[idx];
-    const __nv_bfloat16* w = W + (size_t)t * h;
-    const size_t rp = ((size_t)b * T + pi) * h, rg = ((size_t)b * T + (gp >= 0 ? gp : pi)) * h;
-    for (int i = threadIdx.x; i < h; i += 128) {
-      const float wv = __bfloat162float(w[i]);
-      dp += wv * (__bfloat162float(a_hi[rp + i]) + __bfloat162float(a_lo[rp + i]));
-      dg += wv * (__bfloat162float(a_hi[rg + i]) + __bfloat162float(a_lo[rg + i]));
-    }
-  }
-  for (int o = 16; o > 0; o >>= 1) {
-    dp += __shfl_xor_sync(0xffffffffu, dp, o);
-    dg += __shfl_xor_sync(0xffffffffu, dg, o);
-  }
-  if ((threadIdx.x & 31) == 0) {
-    red[0][threadIdx.x >> 5] = dp;
-    red[1][threadIdx.x >> 5] = dg;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    cand_parent[idx] = pi >= 0 ? red[0][0] + red[0][1] + red[0][2] + red[0][3] : 0.f;
-    cand_gparent[idx] = gp >= 0 ? red[1][0] + red[1][1] + red[1][2] + red[1][3] : 0.f;
-  }
-}
-
 }  // namespace
 
 int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* w_head, const int32_t* tok,
-                     float* logits, float* row_lse, float* cand_parent, float* cand_gparent, cudaStream_t s) {
+                     float* logits, float* cand_parent, float* cand_gparent, cudaStream_t s) {
   const cascade_shape& sh = ctx->shape;
-  const int M = sh.B * tree->T;
+  GemmEpilogue e;
+  e.C = logits;
+  e.ldc = sh.V;
+  e.part = ctx->head_part;
+  e.part_ld = ctx->head_max_tiles;
   if (tok != nullptr) {
-    dim3 grid(tree->T, sh.B);
-    KernelScope ks(ctx, K_CAND_LOGITS, s);
-    k_cand_logits<<<grid, 128, 0, s>>>(ctx->head_a_hi, ctx->head_a_lo, w_head, tree->T, sh.h, sh.V, tok,
-                                       tree->d_parent, cand_parent, cand_gparent);
-    CASCADE_CUDA_TRY(cudaGetLastError());
+    e.tok = tok;
+    e.parent = tree->d_parent;
+    e.T = tree->T;
+    e.n_rows = sh.B * tree->T;
+    e.cand_parent = cand_parent;
+    e.cand_gparent = cand_gparent;
   }
-  return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a_hi, ctx->head_a_lo, M, logits, sh.V, ctx->head_part,
-                        cascade_detail::ceil_div(sh.V, 128), row_lse, K_GEMM_HEAD, s);
+  return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a_hi, ctx->head_lo_offset, sh.B * tree->T, e, K_GEMM_HEAD,
+                        s);
 }
 
 int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const float* gamma, float eps,
                           float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
-                          cudaStream_t s) {
+                          float* cand_parent, float* cand_gparent, cudaStream_t s) {
   const cascade_shape& sh = ctx->shape;
   dim3 grid(T, sh.B);
   KernelScope ks(ctx, K_FINAL_NORM_MIX, s);
   if (sh.dtype == CASCADE_BF16)
-    k_final_norm_mix<__nv_bfloat16><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(hidden), sh.B, T, sh.h,
-                                                         gamma, eps, cfg_scale, inv_temperature, feat, feat_norm,
-                                                         ctx->head_a_hi, ctx->head_a_lo, nullptr);
+    k_final_norm_mix<__nv_bfloat16><<<grid, kNormThreads, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(hidden), sh.B, T, sh.h, gamma, eps, cfg_scale, inv_temperature, feat,
+        feat_norm, ctx->head_a_hi, ctx->head_a_hi + ctx->head_lo_offset, nullptr, cand_parent, cand_gparent);
   else
-    k_final_norm_mix<float><<<grid, 256, 0, s>>>(static_cast<const float*>(hidden), sh.B, T, sh.h, gamma, eps,
-                                                 cfg_scale, inv_temperature, feat, feat_norm, nullptr, nullptr,
-                                                 ctx->head_a_f32);
+    k_final_norm_mix<float><<<grid, kNormThreads, 0, s>>>(static_cast<const float*>(hidden), sh.B, T, sh.h, gamma, eps,
+                                                          cfg_scale, inv_temperature, feat, feat_norm, nullptr,
+                                                          nullptr, ctx->head_a_f32, cand_parent, cand_gparent);
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }

@@ -100,6 +100,21 @@ const CUtensorMap* get_tmap_4d_bf16(cascade_ctx* ctx, const void* base, const ui
   return lookup_or_make(ctx, k);
 }
 
+const CUtensorMap* get_tmap_bf16(cascade_ctx* ctx, const void* base, int rank, const uint64_t* dims,
+                                 const uint64_t* strides_elems, const uint32_t* box) {
+  if (rank < 2 || rank > 4) return nullptr;
+  Key k;
+  std::memset(&k, 0, sizeof(k));
+  k.base = base;
+  k.rank = rank;
+  for (int i = 0; i < rank; ++i) {
+    k.dims[i] = dims[i];
+    k.box[i] = box[i];
+  }
+  for (int i = 0; i + 1 < rank; ++i) k.strides[i] = strides_elems[i];
+  return lookup_or_make(ctx, k);
+}
+
 void free_tmap_cache(cascade_ctx* ctx) {
   delete static_cast<Cache*>(ctx->tmap_cache);
   ctx->tmap_cache = nullptr;

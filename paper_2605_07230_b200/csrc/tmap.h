@@ -14,4 +14,7 @@ const CUtensorMap* get_tmap_2d_bf16(cascade_ctx* ctx, const void* base, uint64_t
 // 4-D map [d3][d2][d1][d0] bf16, d0 contiguous, strides in elements for d1..d3, box sizes per dim.
 const CUtensorMap* get_tmap_4d_bf16(cascade_ctx* ctx, const void* base, const uint64_t dims[4],
                                     const uint64_t strides_elems[3], const uint32_t box[4]);
+// General form: rank 2..4, dims[0] contiguous, strides in elements for dims 1..rank-1.
+const CUtensorMap* get_tmap_bf16(cascade_ctx* ctx, const void* base, int rank, const uint64_t* dims,
+                                 const uint64_t* strides_elems, const uint32_t* box);
 void free_tmap_cache(cascade_ctx* ctx);
