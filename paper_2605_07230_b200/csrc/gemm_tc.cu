@@ -6,25 +6,31 @@
 // dominant cost of verification) and every other projection of the decoder layer.  With M of the
 // order of the draft-tree size the product is bound by streaming W from HBM once, so the kernel is
 // organised around that stream:
-//   * the WEIGHT rows sit on the UMMA M dimension (128 per tile) and the activation rows on the UMMA
-//     N dimension (NB = M rounded up to 16, <= 256), so no tensor-core work is spent on padding a
-//     small M up to 128;
-//   * the work is the flattened list of (weight tile, K block) units, cut into one contiguous,
-//     equally long range per CTA (one CTA per SM), so every SM streams the same number of weight
-//     bytes whatever the number of tiles.  A CTA whose range starts inside a tile adds its partial
-//     accumulator to a scratch slot and raises a flag; the CTA that holds the tile's first K block
-//     reaches that tile last, adds the partials of the CTAs after it in index order (deterministic)
-//     and runs the epilogue.  The launch is cooperative, so all CTAs are resident; the wait is bounded;
-//   * a TMA producer thread keeps a ring of [W 128 x BK | Ahi NB x BK | Alo NB x BK] bf16 stages
+//   * the WEIGHT rows sit on the UMMA M dimension and the activation rows on the UMMA N dimension
+//     (NB = M rounded up to 16, <= 128), so no tensor-core work is spent on padding a small M up to
+//     128.  A work tile is 128 weight rows (kHalves = 1; the kernel also takes 256-row tiles, two
+//     accumulators on one activation stage);
+//   * two ways of spreading the work over the SMs (one CTA per SM):
+//       contiguous (splits = 0): the flattened list of (tile, K block) units is cut into one equally
+//         long range per CTA, so every SM streams the same number of weight bytes whatever the number
+//         of tiles.  A CTA whose range starts inside a tile writes its partial accumulator to a
+//         scratch slot and raises a flag; the CTA that holds the tile's first K block reaches that tile
+//         last, adds the partials of the CTAs after it in index order (deterministic; they were
+//         produced earlier, so they are summed into spare TMEM columns while this CTA's own UMMAs run) and
+//         runs the epilogue.  The launch is cooperative, so all CTAs are resident; the wait is bounded;
+//       sliced (splits = S): K is cut into S slices, work item (tile, slice) writes its own output
+//         matrix and the consumer adds the S matrices.  Nothing waits inside the kernel; this is for
+//         weight matrices with so few tiles that each would be cut many times;
+//   * a TMA producer thread keeps a ring of [W rows x 64 | Ahi NB x 64 | Alo NB x 64] bf16 stages
 //     (128-byte swizzle) in flight, one thread issues the UMMAs (the high part and the remainder of the
 //     activation operand accumulate into the same fp32 TMEM accumulator), and four epilogue warps
-//     drain one of two TMEM accumulators while the next tile is being accumulated into the other.
+//     drain one of two TMEM accumulator sets while the next tile is being accumulated into the other.
 //     The producer and issue loops are kept to a few dozen instructions per stage: a single thread
-//     retires an instruction every few cycles, and at 16 KB of weights per round trip that latency,
-//     not HBM, was the limit;
-//   * epilogue: TMEM lane = weight row n, column = activation row m.  Optional store of (or addition
-//     into) C, coalesced over n; optional per-(m, tile) softmax partials (max, sum of exp) and gather
-//     of the few logits the acceptance rule reads (Algorithm 2: q_x = gtp[x]).
+//     retires an instruction every few cycles, and that latency, not HBM, is the limit otherwise;
+//   * epilogue: TMEM lane = weight row n (within a 128-row tile), column = activation row m.  Optional
+//     store of (or addition into) C, coalesced over n; optional per-(m, tile) softmax partials
+//     (max, sum of exp) and gather of the few logits the acceptance rule reads (Algorithm 2:
+//     q_x = gtp[x]).
 // Every mbarrier / flag wait is bounded; on expiry the CTA records an error word and leaves through
 // the normal teardown (TMEM is freed).
 #include "cascade_internal.h"
@@ -35,17 +41,23 @@
 namespace {
 
 constexpr int kThreads = 192;       // warp 0: TMA, warp 1: UMMA issue + TMEM alloc, warps 2-5: epilogue
-constexpr int kTileN = 128;         // weight rows per tile (UMMA M)
-constexpr int kSpan = 64;           // K elements per 128-byte swizzle span
+constexpr int kTileN = 128;         // weight rows per accumulator (UMMA M)
+constexpr int kSpan = 64;           // K elements per stage (one 128-byte swizzle span)
 constexpr int kMaxStages = 8;
-constexpr int kStRow = 136;         // staging row stride (floats): 136 = 8 mod 32 keeps reads conflict-free
-constexpr int kWSpanBytes = kTileN * kSpan * 2;
+constexpr int kGatherCap = 128;     // candidate logits one 128-row tile can serve from the shared list
+constexpr int kStCols = 32;         // activation rows staged per softmax round
+constexpr int kStRow = 132;         // floats per staged activation row: 4 runs of 33 (32 weight rows + 1 pad)
+constexpr int kTileWBytes = kTileN * kSpan * 2;
 
 struct GemmArgs {
   int M, N, NB, n_mchunks, n_kb, stages, tmem_cols;
-  long long units;      // n_tiles * n_kb
+  int stash;               // 1: TMEM has room for a third accumulator set (partials of split tiles)
+  long long units;         // n_tiles * n_kb
+  int n_tiles;
+  int splits;              // 0: contiguous ranges with in-kernel hand-off; S >= 1: S K slices per tile
+  long long slice_stride;  // floats between the C matrices of consecutive K slices
   GemmEpilogue epi;
-  float* sk_scratch;    // [grid][NB][128] partial accumulators of split tiles
+  float* sk_scratch;       // [grid][halves][NB][128] partial accumulators of split tiles
   unsigned int* sk_flags;
   int* err;
 };
@@ -69,19 +81,34 @@ __device__ __forceinline__ void st_release(unsigned int* p, unsigned int v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-// One contiguous piece of a CTA's range: K blocks [kb0, kb1) of `tile`.
+// One piece of work: K blocks [kb0, kb1) of `tile`; `slice` selects the output matrix in sliced mode.
 struct Segment {
-  int tile, kb0, kb1;
+  int tile, kb0, kb1, slice;
 };
+// Contiguous mode (splits == 0): the flattened (tile, K block) list is cut into one range per CTA and
+// a segment is the part of a tile inside that range.  Sliced mode: work item w = (tile, K slice), taken
+// round-robin by the CTAs.
 struct SegmentWalk {
   long long u, u_end;
-  int n_kb;
-  __device__ SegmentWalk(const GemmArgs& p) : n_kb(p.n_kb) {
+  int n_kb, splits, w, n_items;
+  __device__ SegmentWalk(const GemmArgs& p) : n_kb(p.n_kb), splits(p.splits) {
     u = (long long)blockIdx.x * p.units / gridDim.x;
     u_end = (long long)(blockIdx.x + 1) * p.units / gridDim.x;
+    w = blockIdx.x;
+    n_items = p.n_tiles * p.splits;
   }
   __device__ bool next(Segment& s) {
+    if (splits > 0) {
+      if (w >= n_items) return false;
+      s.tile = w / splits;
+      s.slice = w - s.tile * splits;
+      s.kb0 = (int)((long long)s.slice * n_kb / splits);
+      s.kb1 = (int)((long long)(s.slice + 1) * n_kb / splits);
+      w += gridDim.x;
+      return true;
+    }
     if (u >= u_end) return false;
+    s.slice = 0;
     s.tile = (int)(u / n_kb);
     s.kb0 = (int)(u - (long long)s.tile * n_kb);
     const long long left = u_end - u;
@@ -91,20 +118,25 @@ struct SegmentWalk {
   }
 };
 
-template <int kSpans>
+// kHalves: accumulators (128 weight rows each) per work tile.  kSpans: 64-wide K spans per stage.
+template <int kHalves, int kSpans>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_a, const GemmArgs p) {
+  constexpr int kWSpanBytes = kHalves * kTileWBytes;  // weights of one span
+  constexpr int kWBytes = kSpans * kWSpanBytes;       // weights of one stage: span after span
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ float st[16 * kStRow];
+  __shared__ float st[kStCols * kStRow];
+  __shared__ int s_gather_n;
+  __shared__ int4 s_gather[kGatherCap];  // {weight row in tile, parent column, grandparent column, idx}
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const int a_span_bytes = 2 * p.NB * kSpan * 2;  // hi block then lo block of one span
-  const int stage_bytes = kSpans * (kWSpanBytes + a_span_bytes);
+  const int a_span_bytes = 2 * p.NB * kSpan * 2;  // one span of the activations: hi block then lo block
+  const int stage_bytes = kWBytes + kSpans * a_span_bytes;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
@@ -140,7 +172,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
       Segment sg;
       bool ok = true;
       while (ok && walk.next(sg)) {
-        const int n0 = (sg.tile / n_mchunks) * kTileN, m0 = (sg.tile % n_mchunks) * NB;
+        const int n0 = (sg.tile / n_mchunks) * (kHalves * kTileN), m0 = (sg.tile % n_mchunks) * NB;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
           if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.err)) {
             ok = false;
@@ -149,12 +181,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           uint8_t* stage = smem + s * stage_bytes;
           ptx::mbar_arrive_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
 #pragma unroll
-          for (int q = 0; q < kSpans; ++q)
+          for (int q = 0; q < kSpans; ++q) {
             ptx::tma_load_2d(stage + q * kWSpanBytes, &tm_w, (kb * kSpans + q) * kSpan, n0, &full_bar[s]);
-#pragma unroll
-          for (int q = 0; q < kSpans; ++q)
-            ptx::tma_load_3d(stage + kSpans * kWSpanBytes + q * a_span_bytes, &tm_a, (kb * kSpans + q) * kSpan, m0, 0,
-                             &full_bar[s]);
+            ptx::tma_load_3d(stage + kWBytes + q * a_span_bytes, &tm_a, (kb * kSpans + q) * kSpan, m0, 0, &full_bar[s]);
+          }
           if (++s == stages) {
             s = 0;
             ph ^= 1u;
@@ -178,7 +208,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         ++seg_i;
         if (!ptx::mbar_wait(&tmem_empty[acc], aph ^ 1u, abort_flag, p.err)) break;
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.NB;
+        const uint32_t d_tmem = tmem_base + acc * (uint32_t)(kHalves * p.NB);
         uint32_t accumulate = 0;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
           if (!ptx::mbar_wait(&full_bar[s], ph, abort_flag, p.err)) {
@@ -187,19 +217,22 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           }
           ptx::tc_fence_after();
           const uint32_t w_addr = smem_base + (uint32_t)(s * stage_bytes);
-          const uint32_t a_addr = w_addr + kSpans * kWSpanBytes;
 #pragma unroll
           for (int q = 0; q < kSpans; ++q) {
-            const uint64_t wd0 = ptx::umma_desc_sw128(w_addr + q * kWSpanBytes);
-            const uint64_t ad0 = ptx::umma_desc_sw128(a_addr + q * a_span_bytes);
+            const uint64_t ad0 = ptx::umma_desc_sw128(w_addr + kWBytes + q * a_span_bytes);
 #pragma unroll
-            for (int ks = 0; ks < kSpan / 16; ++ks) {
-              // advancing 16 K elements = 32 bytes = 2 descriptor units inside the swizzle span
-              ptx::umma_bf16(d_tmem, wd0 + 2 * ks, ad0 + 2 * ks, idesc, accumulate);
-              accumulate = 1u;
-              ptx::umma_bf16(d_tmem, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
+            for (int t = 0; t < kHalves; ++t) {
+              const uint64_t wd0 = ptx::umma_desc_sw128(w_addr + q * kWSpanBytes + t * kTileWBytes);
+              const uint32_t d = d_tmem + t * (uint32_t)p.NB;
+#pragma unroll
+              for (int ks = 0; ks < kSpan / 16; ++ks) {
+                // advancing 16 K elements = 32 bytes = 2 descriptor units inside the swizzle span
+                ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + 2 * ks, idesc, (q | ks) == 0 ? accumulate : 1u);
+                ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
+              }
             }
           }
+          accumulate = 1u;
           ptx::umma_commit(&empty_bar[s]);  // stage reusable once these UMMAs have read it
           if (++s == stages) {
             s = 0;
@@ -215,7 +248,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     const int quad = warp & 3;                  // TMEM lane quadrant this warp may read
     const int vl = quad * 32 + lane;            // weight row within the tile
     const int eid = (warp - 2) * 32 + lane;     // 0..127
-    const int st_m = eid >> 3, st_part = eid & 7;
+    const int st_col = eid >> 2, st_part = eid & 3;  // softmax round: 4 threads per staged activation row
+    const int st_wr = (vl >> 5) * 33 + (vl & 31);    // where this thread's weight row goes in a staged row
     const GemmEpilogue& e = p.epi;
     const int NB = p.NB;
     uint32_t seg_i = 0;
@@ -224,11 +258,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     while (walk.next(sg)) {
       const uint32_t acc = seg_i & 1u, aph = (seg_i >> 1) & 1u;
       ++seg_i;
-      const int n_tile = sg.tile / p.n_mchunks;
-      const int n = n_tile * kTileN + vl, m0 = (sg.tile % p.n_mchunks) * NB;
-      const bool contributor = sg.kb0 > 0;
-      const bool owner_of_split = sg.kb0 == 0 && sg.kb1 < p.n_kb;
+      const int macro = sg.tile / p.n_mchunks, m0 = (sg.tile % p.n_mchunks) * NB;
+      const bool contributor = p.splits == 0 && sg.kb0 > 0;
+      const bool owner_of_split = p.splits == 0 && sg.kb0 == 0 && sg.kb1 < p.n_kb;
+      float* const c_out = e.C != nullptr ? e.C + (size_t)sg.slice * p.slice_stride : nullptr;
       int n_contrib = 0;
+      bool presummed = false;
+      // spare TMEM columns behind the two accumulator sets hold the sum of the other CTAs' partials
+      const uint32_t stash_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(2 * kHalves * NB);
       if (owner_of_split) {
         // the CTAs after this one whose range starts inside this tile each hold one partial of it
         const long long tile_end = (long long)(sg.tile + 1) * p.n_kb;
@@ -249,69 +286,161 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           }
         }
         ptx::named_bar_sync(1, 128);
+        if (*abort_flag) break;
+        if (p.stash) {
+          // they finished their piece earlier: add them up now, while this CTA's own UMMAs are running
+          presummed = true;
+          for (int c = 0; c < kHalves * NB; c += 16) {  // column c of the [half][NB] slot layout
+            float acc16[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc16[i] = 0.f;
+            for (int k = 1; k <= n_contrib; ++k) {
+              const float* slot = p.sk_scratch + ((size_t)(blockIdx.x + k) * (kHalves * NB) + c) * kTileN + vl;
+              float t[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) t[i] = __ldcg(slot + (size_t)i * kTileN);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) acc16[i] += t[i];
+            }
+            ptx::tmem_st16(stash_addr + c, acc16);
+          }
+        }
       }
-      if (*abort_flag) break;
       if (!ptx::mbar_wait(&tmem_full[acc], aph, abort_flag, p.err)) break;
       ptx::tc_fence_after();
-      const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * (uint32_t)NB;
-      for (int c0 = 0; c0 < NB; c0 += 16) {
-        float v[16];
-        ptx::tmem_ld16(t_addr + c0, v);
-        if (contributor) {
-          float* slot = p.sk_scratch + ((size_t)blockIdx.x * NB + c0) * kTileN + vl;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) slot[(size_t)i * kTileN] = v[i];
-          continue;
+      for (int half = 0; half < kHalves; ++half) {
+        const int n_tile = macro * kHalves + half;
+        if (n_tile * kTileN >= p.N) break;  // second half of the last work tile lies beyond N
+        const int n = n_tile * kTileN + vl;
+        const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (acc * kHalves + half) * (uint32_t)NB;
+        int n_gather = 0;
+        if (e.tok != nullptr && !contributor) {
+          // which of the logits the acceptance rule reads (tok[idx] under its parent's and grandparent's
+          // rows) fall into this 128-row tile: found once here, served from the staging buffer below
+          ptx::named_bar_sync(1, 128);
+          if (eid == 0) s_gather_n = 0;
+          ptx::named_bar_sync(1, 128);
+          for (int idx = eid; idx < e.n_rows; idx += 128) {
+            const int ln = e.tok[idx] - n_tile * kTileN;
+            if ((unsigned)ln >= (unsigned)kTileN) continue;
+            const int b = idx / e.T, j = idx - b * e.T;
+            const int pi = e.parent[j];
+            if (pi < 0) continue;
+            const int gp = e.parent[pi];
+            const int pos = atomicAdd(&s_gather_n, 1);
+            if (pos < kGatherCap)
+              s_gather[pos] = make_int4((ln >> 5) * 33 + (ln & 31), b * e.T + pi - m0, gp >= 0 ? b * e.T + gp - m0 : -1, idx);
+          }
+          ptx::named_bar_sync(1, 128);
+          n_gather = s_gather_n;
         }
-        for (int k = 1; k <= n_contrib; ++k) {
-          const float* slot = p.sk_scratch + ((size_t)(blockIdx.x + k) * NB + c0) * kTileN + vl;
+        // 64 accumulator columns at a time (NB is a multiple of 16, so the last group may be narrower)
+        for (int c0 = 0; c0 < NB; c0 += 64) {
+          const int n_cols = min(64, NB - c0);
+          float v[64];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] += __ldcg(slot + (size_t)i * kTileN);
-        }
-        if (e.C != nullptr && n < p.N) {
+          for (int sub = 0; sub < 4; ++sub)
+            if (16 * sub < n_cols) ptx::tmem_ld16(t_addr + c0 + 16 * sub, v + 16 * sub);
+          if (contributor) {
+            // partial of a split tile, [column][weight row]: coalesced over the lanes
+            float* slot = p.sk_scratch + (((size_t)blockIdx.x * kHalves + half) * NB + c0) * kTileN + vl;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int m = m0 + c0 + i;
-            if (m < p.M) {
-              float* dst = e.C + (size_t)m * e.ldc + n;
-              *dst = e.accumulate ? *dst + v[i] : v[i];
+            for (int i = 0; i < 64; ++i)
+              if (i < n_cols) slot[(size_t)i * kTileN] = v[i];
+            continue;
+          }
+          if (presummed) {
+#pragma unroll
+            for (int sub = 0; sub < 4; ++sub)
+              if (16 * sub < n_cols) {
+                float t[16];
+                ptx::tmem_ld16(stash_addr + half * NB + c0 + 16 * sub, t);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[16 * sub + i] += t[i];
+              }
+          } else {
+            for (int k = 1; k <= n_contrib; ++k) {
+              const float* slot = p.sk_scratch + (((size_t)(blockIdx.x + k) * kHalves + half) * NB + c0) * kTileN + vl;
+#pragma unroll
+              for (int q = 0; q < 2; ++q) {
+                float t[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (32 * q + i < n_cols) t[i] = __ldcg(slot + (size_t)(32 * q + i) * kTileN);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (32 * q + i < n_cols) v[32 * q + i] += t[i];
+              }
             }
           }
-        }
-        if (e.part != nullptr) {
-          ptx::named_bar_sync(1, 128);  // the previous chunk has been read
+          if (c_out != nullptr && n < p.N) {
+            float* dst = c_out + (size_t)(m0 + c0) * e.ldc + n;
+            const int rows = min(n_cols, p.M - (m0 + c0));  // rows of this group that exist
+            if (e.accumulate) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) st[i * kStRow + vl] = (n < p.N) ? v[i] : -INFINITY;
-          ptx::named_bar_sync(1, 128);
-          float mx = -INFINITY;
+              for (int i = 0; i < 64; ++i)
+                if (i < rows) dst[(size_t)i * e.ldc] += v[i];
+            } else {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) mx = fmaxf(mx, st[st_m * kStRow + st_part + 8 * i]);
-          float sum = 0.f;
-          if (mx != -INFINITY) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) sum += __expf(st[st_m * kStRow + st_part + 8 * i] - mx);
+              for (int i = 0; i < 64; ++i)
+                if (i < rows) dst[(size_t)i * e.ldc] = v[i];
+            }
           }
+          if (e.part != nullptr) {
+            // per-(activation row, tile) softmax partials: 32 activation rows per round go through shared
+            // memory so that 4 threads see the 128 weight rows of one activation row
 #pragma unroll
-          for (int o = 1; o < 8; o <<= 1) {
-            const float mo = __shfl_xor_sync(0xffffffffu, mx, o), so = __shfl_xor_sync(0xffffffffu, sum, o);
-            combine_ms(mx, sum, mo, so);
-          }
-          const int m = m0 + c0 + st_m;
-          if (st_part == 0 && m < p.M) e.part[(size_t)m * e.part_ld + n_tile] = make_float2(mx, sum);
-          if (e.tok != nullptr) {
-            // logits the acceptance rule reads: tok[idx] under its parent's and grandparent's rows
-            for (int idx = eid; idx < e.n_rows; idx += 128) {
-              const int ln = e.tok[idx] - n_tile * kTileN;
-              if ((unsigned)ln >= (unsigned)kTileN) continue;
-              const int b = idx / e.T, j = idx - b * e.T;
-              const int pi = e.parent[j];
-              if (pi < 0) continue;
-              int col = b * e.T + pi - m0 - c0;
-              if ((unsigned)col < 16u) e.cand_parent[idx] = st[col * kStRow + ln];
-              const int gp = e.parent[pi];
-              if (gp < 0) continue;
-              col = b * e.T + gp - m0 - c0;
-              if ((unsigned)col < 16u) e.cand_gparent[idx] = st[col * kStRow + ln];
+            for (int r = 0; r < 2; ++r) {
+              if (r * kStCols >= n_cols) break;
+              const int cs = c0 + r * kStCols;  // first activation row (column) of this round
+              ptx::named_bar_sync(1, 128);      // the previous round has been read
+#pragma unroll
+              for (int i = 0; i < kStCols; ++i)
+                if (r * kStCols + i < n_cols) st[i * kStRow + st_wr] = (n < p.N) ? v[r * kStCols + i] : -INFINITY;
+              ptx::named_bar_sync(1, 128);
+              const float* row = st + st_col * kStRow + st_part * 33;
+              float mx = row[0];
+#pragma unroll
+              for (int i = 1; i < 32; ++i) mx = fmaxf(mx, row[i]);
+              float sum = 0.f;
+              if (mx != -INFINITY) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) sum += __expf(row[i] - mx);
+              }
+#pragma unroll
+              for (int o = 1; o < 4; o <<= 1) {
+                const float mo = __shfl_xor_sync(0xffffffffu, mx, o), so = __shfl_xor_sync(0xffffffffu, sum, o);
+                combine_ms(mx, sum, mo, so);
+              }
+              const int m = m0 + cs + st_col;
+              if (st_part == 0 && r * kStCols + st_col < n_cols && m < p.M)
+                e.part[(size_t)m * e.part_ld + n_tile] = make_float2(mx, sum);
+              if (n_gather <= kGatherCap) {
+                for (int i = eid; i < n_gather; i += 128) {
+                  const int4 g = s_gather[i];
+                  int col = g.y - cs;
+                  if ((unsigned)col < (unsigned)kStCols) e.cand_parent[g.w] = st[col * kStRow + g.x];
+                  col = g.z - cs;
+                  if (g.z >= 0 && (unsigned)col < (unsigned)kStCols) e.cand_gparent[g.w] = st[col * kStRow + g.x];
+                }
+              } else {
+                // more hits in one tile than the list holds: scan the tokens again in every round
+                for (int idx = eid; idx < e.n_rows; idx += 128) {
+                  const int ln = e.tok[idx] - n_tile * kTileN;
+                  if ((unsigned)ln >= (unsigned)kTileN) continue;
+                  const int b = idx / e.T, j = idx - b * e.T;
+                  const int pi = e.parent[j];
+                  if (pi < 0) continue;
+                  const int at = (ln >> 5) * 33 + (ln & 31);
+                  int col = b * e.T + pi - m0 - cs;
+                  if ((unsigned)col < (unsigned)kStCols) e.cand_parent[idx] = st[col * kStRow + at];
+                  const int gp = e.parent[pi];
+                  if (gp < 0) continue;
+                  col = b * e.T + gp - m0 - cs;
+                  if ((unsigned)col < (unsigned)kStCols) e.cand_gparent[idx] = st[col * kStRow + at];
+                }
+              }
             }
           }
         }
@@ -340,51 +469,80 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 
 }  // namespace
 
-int64_t gemm_tc_scratch_floats(int sm_count) { return (int64_t)sm_count * 256 * kTileN; }
+int64_t gemm_tc_scratch_floats(int sm_count) { return (int64_t)sm_count * 2 * 128 * kTileN; }
+
+int gemm_tc_pick_splits(int sm_count, int N, int K, int max_splits) {
+  const int n_tiles = cascade_detail::ceil_div(N, kTileN), n_kb = cascade_detail::ceil_div(K, kSpan);
+  int best = 1;
+  long long best_cost = -1;
+  for (int s = 1; s <= max_splits && s <= n_kb; ++s) {
+    // time ~ rounds x K blocks per item, plus a little per slice for writing and re-reading its matrix
+    const long long rounds = cascade_detail::ceil_div(n_tiles * s, sm_count);
+    const long long cost = rounds * cascade_detail::ceil_div(n_kb, s) * 8 + s;
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = s;
+    }
+  }
+  return best;
+}
 
 int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* a_hi,
                    int64_t lo_offset, int M, const GemmEpilogue& epi, int kernel_id, cudaStream_t s) {
   if (K % 8 != 0 || M < 1 || N < 1 || lo_offset % 8 != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (epi.part != nullptr && epi.part_ld < cascade_detail::ceil_div(N, kTileN)) return CASCADE_ERR_INVALID_ARG;
+  if (epi.splits < 0 || (epi.splits > 1 && (epi.part != nullptr || epi.accumulate || epi.C == nullptr)))
+    return CASCADE_ERR_INVALID_ARG;
   if (epi.tok != nullptr && (epi.part == nullptr || epi.parent == nullptr || epi.cand_parent == nullptr ||
                              epi.cand_gparent == nullptr || epi.T < 1))
     return CASCADE_ERR_INVALID_ARG;
   GemmArgs a;
   a.M = M;
   a.N = N;
-  a.NB = M <= 256 ? (int)cascade_detail::align_up(M, 16) : 128;
-  a.n_mchunks = cascade_detail::ceil_div(M, a.NB);
+  a.n_mchunks = cascade_detail::ceil_div(M, 128);
+  a.NB = (int)cascade_detail::align_up(cascade_detail::ceil_div(M, a.n_mchunks), 16);
   a.epi = epi;
   a.sk_scratch = ctx->gemm_scratch;
   a.sk_flags = ctx->gemm_flags;
   a.err = ctx->dev_error;
-  const int budget = 227 * 1024 - 12 * 1024 - 1024;  // static shared + alignment slack
-  // two swizzle spans per stage when at least three such stages fit, else one
-  const int stage1 = kWSpanBytes + 2 * a.NB * kSpan * 2;
-  const int spans = (budget / (2 * stage1) >= 3) ? 2 : 1;
-  const int stage_bytes = spans * stage1;
+  // A stage carries 32 KB of weights where three such stages fit (two K spans of a 128-row tile): the
+  // round trip of the single producer / issue threads per stage limits the stream below that.  With
+  // many activation rows the activation part of a stage is too large for that: one span per stage.
+  // (256-row tiles -- two accumulators per activation stage, half the activation traffic -- measured
+  // no faster on the stream and split the LM head of a 16384-token vocabulary over too few tiles.)
+  const int halves = 1;
+  const int budget = 227 * 1024 - 20 * 1024 - 1024;  // static shared + alignment slack
+  const int span_bytes = halves * kTileWBytes + 2 * a.NB * kSpan * 2;
+  const int spans = budget / (2 * span_bytes) >= 3 ? 2 : 1;
+  const int stage_bytes = spans * span_bytes;
   a.stages = budget / stage_bytes;
   if (a.stages > kMaxStages) a.stages = kMaxStages;
   if (a.stages < 2) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   a.n_kb = cascade_detail::ceil_div(K, kSpan * spans);
-  const int n_tiles = cascade_detail::ceil_div(N, kTileN) * a.n_mchunks;
+  const int n_tiles = cascade_detail::ceil_div(N, halves * kTileN) * a.n_mchunks;
   a.units = (long long)n_tiles * a.n_kb;
+  a.n_tiles = n_tiles;
+  a.splits = epi.splits;
+  a.slice_stride = epi.slice_stride;
+  a.stash = epi.splits == 0 && 3 * halves * a.NB <= 512;
   a.tmem_cols = 32;
-  while (a.tmem_cols < 2 * a.NB) a.tmem_cols *= 2;
-  const CUtensorMap* tw = get_tmap_2d_bf16(ctx, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileN, kSpan);
+  while (a.tmem_cols < (a.stash ? 3 : 2) * halves * a.NB) a.tmem_cols *= 2;
+  const CUtensorMap* tw =
+      get_tmap_2d_bf16(ctx, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(halves * kTileN), kSpan);
   const uint64_t ad[3] = {(uint64_t)K, (uint64_t)M, 2};
   const uint64_t as[2] = {(uint64_t)K, (uint64_t)lo_offset};
   const uint32_t ab[3] = {kSpan, (uint32_t)a.NB, 2};
   const CUtensorMap* ta = get_tmap_bf16(ctx, a_hi, 3, ad, as, ab);
   if (tw == nullptr || ta == nullptr) return CASCADE_ERR_CUDA;
   const int smem = a.stages * stage_bytes + 1024;
-  auto kern = spans == 2 ? k_gemm_tc<2> : k_gemm_tc<1>;
+  auto kern = spans == 2 ? k_gemm_tc<1, 2> : k_gemm_tc<1, 1>;
   static int configured_smem[2] = {0, 0};
   if (smem > configured_smem[spans - 1]) {
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     configured_smem[spans - 1] = smem;
   }
-  long long grid = a.units < ctx->sm_count ? a.units : ctx->sm_count;
+  long long grid = epi.splits > 0 ? (long long)n_tiles * epi.splits : a.units;
+  if (grid > ctx->sm_count) grid = ctx->sm_count;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(kThreads);
@@ -394,7 +552,7 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident: the split-tile hand-off waits on peers
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = epi.splits == 0 ? 1 : 0;
   {
     KernelScope ks(ctx, kernel_id, s);
     CASCADE_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, *tw, *ta, a));

@@ -6,6 +6,12 @@ struct GemmEpilogue {
   float* C = nullptr;      // [M][ldc] fp32 result
   int ldc = 0;
   int accumulate = 0;      // 1: C += result (residual add), 0: C = result
+  // splits = 0: the kernel balances (tile, K block) work over the SMs and adds the pieces of a tile
+  // itself.  splits = S >= 1: K is cut into S slices and slice s writes its own matrix
+  // C + s * slice_stride; the consumer adds the S matrices (no waiting inside the kernel; S > 1 needs C,
+  // no accumulate, no part).
+  int splits = 0;
+  int64_t slice_stride = 0;
   float2* part = nullptr;  // per-(row, 128-wide tile) softmax partials (max, sum of exp): part[m * part_ld + tile]
   int part_ld = 0;
   // gather of the logits the acceptance rule reads (needs part): for idx = b * T + j,
@@ -24,3 +30,5 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
                    int64_t lo_offset, int M, const GemmEpilogue& epi, int kernel_id, cudaStream_t s);
 // Floats of scratch the split-tile hand-off needs for a device with `sm_count` SMs.
 int64_t gemm_tc_scratch_floats(int sm_count);
+// Number of K slices (splits >= 1) that keeps the SMs evenly busy for an [N][K] weight matrix.
+int gemm_tc_pick_splits(int sm_count, int N, int K, int max_splits);

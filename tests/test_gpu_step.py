@@ -37,7 +37,10 @@ def check_step(wl: PiecesWorkload, s, mode, flags):
     # end to end (checker from the raw inputs): reported, and expected to agree except at near ties
     full = [O.relaxed_accept(ref_head["feat"][b], ref_head["logits"][b], h["tok"][b], parent, h["draft_p"][b],
                              h["uniforms"][b], w.tau_pos, w.tau_seq, w.tvd_budget, flags) for b in range(w.B)]
-    agree = np.mean([np.array_equal(full[b]["accept"], s.out["accept"].cpu().numpy()[b]) for b in range(w.B)])
+    # fraction of nodes on which the two accept masks agree (a score inside the near band, or a logit
+    # that differs in its last bits, may flip a node: reported, with a loose floor)
+    got = s.out["accept"].cpu().numpy()
+    agree = np.mean([np.mean(full[b]["accept"] == got[b]) for b in range(w.B)])
     return st, agree, rows
 
 
@@ -62,7 +65,7 @@ def test_fused_step(name, over, mode):
         agree.append(a)
     assert compared >= 1
     assert relaxed > 0                      # the relaxation took part in these decisions
-    assert np.mean(agree) >= 0.5
+    assert np.mean(agree) >= 0.9
     assert wl.ctx.last_launch_count >= 5
     wl.close()
 
