@@ -85,7 +85,7 @@ __device__ __forceinline__ int sib_pair_index(int x, int y, int k) { return x * 
 
 // ---- the rule: whole CTA (kTailThreads threads), one prompt ------------------------------------------
 __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
-  __shared__ int32_t s_parent[kMaxT], s_depth[kMaxT], s_cb[kMaxT], s_cc[kMaxT], s_tok[kMaxT];
+  __shared__ int32_t s_parent[kMaxT], s_depth[kMaxT], s_cb[kMaxT], s_cc[kMaxT], s_tok[kMaxT], s_sib[kMaxT];
   __shared__ float s_q[kMaxT];    // mass of tok[j] under its parent's row
   __shared__ float s_qg[kMaxT];   // mass of tok[j] under its grandparent's row
   __shared__ float s_lse[kMaxT], s_mI[kMaxT], s_mC[kMaxT], s_qR[kMaxT], s_tvd[kMaxT];
@@ -100,16 +100,23 @@ __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
   const size_t row0 = (size_t)b * T;
   const cascade_params prm = io.prm;
   for (int i = j; i < tr.n_pairs; i += kTailThreads) s_scores[i] = __ldcg(io.scores + (size_t)b * tr.n_pairs + i);
-  float my_p = 0.f, my_u = 1.f;
+  // every global read of this block is issued here, in one round trip
+  float my_p = 0.f, my_u = 1.f, my_cp = 0.f, my_cg = 0.f;
+  uint64_t my_anc[kMaxT / 64] = {0, 0, 0, 0};
   if (j < T) {
     s_parent[j] = tr.parent[j];
     s_depth[j] = tr.depth[j];
     s_cb[j] = tr.child_begin[j];
     s_cc[j] = tr.child_count[j];
+    s_sib[j] = tr.sib_base[j];
     s_tok[j] = io.tok[row0 + j];
     s_lse[j] = __ldcg(io.row_lse + row0 + j);
     my_p = io.draft_p[row0 + j];
     my_u = io.uniforms[row0 + j];
+    my_cp = __ldcg(io.cand_parent + row0 + j);
+    my_cg = __ldcg(io.cand_gparent + row0 + j);
+#pragma unroll
+    for (int w = 0; w < kMaxT / 64; ++w) my_anc[w] = tr.anc[(size_t)j * 4 + w];
   }
   __syncthreads();
   // 1. target mass of each drafted token under its parent's (and grandparent's) distribution
@@ -117,8 +124,8 @@ __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
     float q = 0.f, qg = 0.f;
     if (j >= 1) {
       const int pi = s_parent[j];
-      q = expf(__ldcg(io.cand_parent + row0 + j) - s_lse[pi]);
-      if (s_parent[pi] >= 0) qg = expf(__ldcg(io.cand_gparent + row0 + j) - s_lse[s_parent[pi]]);
+      q = expf(my_cp - s_lse[pi]);
+      if (s_parent[pi] >= 0) qg = expf(my_cg - s_lse[s_parent[pi]]);
     }
     s_q[j] = q;
     s_qg[j] = qg;
@@ -132,7 +139,7 @@ __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
     uint32_t imask = 0, near = 0;
     float mI = 0.f, mC = 0.f;
     if (prm.flags & CASCADE_USE_I) {
-      const int base = tr.sib_base[pi];
+      const int base = s_sib[pi];
       for (int s = 0; s < k; ++s) {
         if (s == me) continue;
         const float c = s_scores[base + (s < me ? sib_pair_index(s, me, k) : sib_pair_index(me, s, k))];
@@ -248,9 +255,9 @@ __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
   uint32_t key = 0;  // (depth, smallest index first) of a node whose whole path is covered
   if (j < T) {
     bool on_path = true;
-    const uint64_t* anc = tr.anc + (size_t)j * 4;
-    for (int w = 0; w < (T + 63) / 64; ++w) {
-      const uint64_t need = anc[w];
+#pragma unroll
+    for (int w = 0; w < kMaxT / 64; ++w) {
+      const uint64_t need = my_anc[w];
       const uint64_t have = (uint64_t)cover[2 * w] | ((uint64_t)cover[2 * w + 1] << 32);
       if (need & ~have) on_path = false;
     }
@@ -321,15 +328,29 @@ __global__ void __launch_bounds__(kTailThreads) k_tail(const TreeDev tr, const T
     const int row = (blk - n_pair_blocks) * (kTailThreads / 32) + warp;
     if (row < tr.T) {
       const float2* pr = ta.part + ((size_t)b * tr.T + row) * ta.part_ld;
-      float mx = -INFINITY;
-      for (int t = lane; t < ta.n_tiles; t += 32) mx = fmaxf(mx, __ldcg(&pr[t]).x);
-      mx = warp_max(mx);
-      float sum = 0.f;
-      for (int t = lane; t < ta.n_tiles; t += 32) {
-        const float2 ms = __ldcg(&pr[t]);
-        if (ms.x != -INFINITY) sum += ms.y * __expf(ms.x - mx);
+      // 16 partials per lane per round, all loads of a round in flight together
+      float mx = -INFINITY, sum = 0.f;
+      for (int t0 = 0; t0 < ta.n_tiles; t0 += 32 * 16) {
+        float2 ms[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int t = t0 + i * 32 + lane;
+          ms[i] = t < ta.n_tiles ? __ldcg(&pr[t]) : make_float2(-INFINITY, 0.f);
+        }
+        float m2 = mx;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) m2 = fmaxf(m2, ms[i].x);
+        if (m2 != -INFINITY) {
+          sum *= __expf(mx - m2);
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            if (ms[i].x != -INFINITY) sum += ms[i].y * __expf(ms[i].x - m2);
+        }
+        mx = m2;
       }
-      sum = warp_sum(sum);
+      const float m_all = warp_max(mx);
+      sum = warp_sum(mx == -INFINITY ? 0.f : sum * __expf(mx - m_all));
+      mx = m_all;
       if (lane == 0) ta.row_lse_out[(size_t)b * tr.T + row] = mx + logf(sum);
     }
   }

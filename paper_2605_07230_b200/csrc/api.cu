@@ -49,6 +49,7 @@ int64_t carve(cascade_ctx* c, char* base) {
   const int t_pad = (int)align_up(T, 64);
   cv.take(c->attn_part_o, (int64_t)R * s.Hq * c->attn_max_splits * t_pad * s.D);
   cv.take(c->attn_part_ml, (int64_t)R * s.Hq * c->attn_max_splits * t_pad);
+  cv.take(c->attn_unit_done, (int64_t)R * s.Hq * (t_pad / 64));
   c->head_m_pad = (int)align_up(BT, 128);
   if (s.dtype == CASCADE_BF16) {
     c->head_lo_offset = (int64_t)c->head_m_pad * s.h;
@@ -111,7 +112,7 @@ const char* cascade_strerror(int status) {
 }
 
 const char* cascade_kernel_name(int32_t id) {
-  static const char* names[] = {"tree_attn", "attn_combine", "tree_attn_f32", "final_norm_mix", "gemm_head",
+  static const char* names[] = {"tree_attn", "tree_attn_f32", "final_norm_mix", "gemm_head",
                                 "head_f32", "row_stats", "row_lse", "similarity", "accept", "tail", "select_path",
                                 "embed_norm", "gemm_qkv", "rope_split", "gemm_o", "resid_norm", "gemm_gate_up",
                                 "swiglu", "gemm_down", "gemm_f32", "resid_add"};

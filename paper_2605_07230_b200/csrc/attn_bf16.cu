@@ -16,8 +16,9 @@
 //   * keys of the prefix are visible to every row up to prefix_len; keys of the tree are visible to
 //     row j iff bit i of the packed ancestor-or-self mask of j is set (one 64-bit word per lane and
 //     tile half).
-// With several KV splits each CTA writes an un-normalised partial (output, max, sum) and a second
-// small kernel merges them; with one split the CTA writes the final bf16 rows itself.
+// With several KV splits each CTA writes an un-normalised partial (output, max, sum); the CTA of a
+// (CFG row, head, row block) that finishes last merges them in split order (a counter per unit, no
+// waiting) and writes the bf16 rows.  With one split the CTA writes the final rows itself.
 // Every mbarrier wait is bounded (error word + normal teardown on expiry).
 #include "cascade_internal.h"
 #include "ptx.cuh"
@@ -46,6 +47,7 @@ struct AttnArgs {
   float2* part_ml;
   float c;  // softmax_scale * log2(e)
   int* err;
+  unsigned int* unit_done;  // [R * Hq * n_rb] finished-split counters, zero between launches
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -56,7 +58,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   __shared__ __align__(8) uint64_t q_full, kv_full[kStages], kv_empty[kStages], s_full[2], s_empty[2], p_full,
       o_full[2], o_empty[2];
   __shared__ uint32_t s_tmem_base;
-  __shared__ int s_abort;
+  __shared__ int s_abort, s_last;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -321,25 +323,54 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, 512);
   }
-}
-
-// Merge of the split-KV partials: out = sum_s w_s O_s / sum_s w_s l_s, w_s = 2^(m_s - max m).
-__global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ part_o,
-                                                      const float2* __restrict__ part_ml, int T, int Hq, int splits,
-                                                      int t_pad, __nv_bfloat16* __restrict__ out) {
-  const int j = blockIdx.x, head = blockIdx.y, r = blockIdx.z, d = threadIdx.x;
-  const size_t unit0 = ((size_t)r * Hq + head) * splits;
+  if (p.splits == 1) return;
+  // ---- the last split of this (CFG row, head, row block) to finish merges all of them ----
+  const unsigned int unit_id = ((unsigned)r * p.Hq + head) * p.n_rb + rb;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned int ticket = atomicAdd(p.unit_done + unit_id, 1u);
+    s_last = ticket == (unsigned)p.splits - 1;
+    if (s_last) p.unit_done[unit_id] = 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (threadIdx.x >= 128) return;
+  // out = sum_s w_s O_s / sum_s w_s l_s, w_s = 2^(m_s - max m), splits taken in index order
+  const int row = threadIdx.x & 63, j = rb * kRowsPerBlock + row, d0 = (threadIdx.x >> 6) * (kD / 2);
+  if (j >= p.T) return;
+  const size_t unit0 = ((size_t)r * p.Hq + head) * p.splits;
   float m = -INFINITY;
-  for (int s = 0; s < splits; ++s) m = fmaxf(m, part_ml[(unit0 + s) * t_pad + j].x);
-  float acc = 0.f, l = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    const float2 ml = part_ml[(unit0 + s) * t_pad + j];
+  for (int s = 0; s < p.splits; ++s) m = fmaxf(m, __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + j]).x);
+  float acc[kD / 2];
+#pragma unroll
+  for (int d = 0; d < kD / 2; ++d) acc[d] = 0.f;
+  float l = 0.f;
+  for (int s = 0; s < p.splits; ++s) {
+    const float2 ml = __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + j]);
     if (ml.x == -INFINITY) continue;
     const float w = ptx::ex2(ml.x - m);
-    acc += w * part_o[((unit0 + s) * t_pad + j) * kD + d];
     l += w * ml.y;
+    const float4* src = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s) * p.t_pad + j) * kD + d0);
+#pragma unroll
+    for (int c = 0; c < kD / 8; ++c) {
+      const float4 t = __ldcg(src + c);
+      acc[4 * c] += w * t.x;
+      acc[4 * c + 1] += w * t.y;
+      acc[4 * c + 2] += w * t.z;
+      acc[4 * c + 3] += w * t.w;
+    }
   }
-  out[(((size_t)r * T + j) * Hq + head) * kD + d] = __float2bfloat16_rn(acc / l);
+  const float inv = 1.f / l;
+  uint4* dst = reinterpret_cast<uint4*>(p.out + (((size_t)r * p.T + j) * p.Hq + head) * kD + d0);
+#pragma unroll
+  for (int c = 0; c < kD / 16; ++c) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) w[k] = ptx::pack_bf16x2(acc[8 * c + 2 * k] * inv, acc[8 * c + 2 * k + 1] * inv);
+    dst[c] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
 }
 
 }  // namespace
@@ -365,10 +396,11 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   a.part_ml = ctx->attn_part_ml;
   a.c = scale * 1.4426950408889634f;
   a.err = ctx->dev_error;
-  // KV splits: enough CTAs to cover the SMs, never more splits than tiles, never more than the scratch holds
+  a.unit_done = ctx->attn_unit_done;
+  // KV splits: as many as fit on the SMs at once, never more splits than tiles or than the scratch holds
   const int n_tiles = cascade_detail::ceil_div(prefix_cap, kTileKeys) + cascade_detail::ceil_div(T, kTileKeys);
   const int units = R * sh.Hq * a.n_rb;
-  int splits = cascade_detail::ceil_div(ctx->sm_count, units);
+  int splits = ctx->sm_count / units;
   if (splits > n_tiles) splits = n_tiles;
   if (splits > ctx->attn_max_splits) splits = ctx->attn_max_splits;
   if (splits < 1) splits = 1;
@@ -403,11 +435,5 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
     k_tree_attn_bf16<<<grid, kThreads, kSmemBytes, s>>>(*mq, *mkp, *mvp, *mkt, *mvt, a);
   }
   CASCADE_CUDA_TRY(cudaGetLastError());
-  if (splits > 1) {
-    dim3 g2(T, sh.Hq, R);
-    KernelScope ks(ctx, K_ATTN_COMBINE, s);
-    k_attn_combine<<<g2, kD, 0, s>>>(ctx->attn_part_o, ctx->attn_part_ml, T, sh.Hq, splits, a.t_pad, out);
-    CASCADE_CUDA_TRY(cudaGetLastError());
-  }
   return CASCADE_OK;
 }

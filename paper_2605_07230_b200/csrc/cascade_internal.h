@@ -32,7 +32,7 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // Kernel ids for the per-kernel timing table.
 enum KernelId : int {
-  K_TREE_ATTN = 0, K_ATTN_COMBINE, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_GEMM_HEAD, K_HEAD_F32, K_ROW_STATS,
+  K_TREE_ATTN = 0, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_GEMM_HEAD, K_HEAD_F32, K_ROW_STATS,
   K_ROW_LSE, K_SIMILARITY, K_ACCEPT, K_TAIL, K_SELECT_PATH, K_EMBED_NORM, K_GEMM_QKV, K_ROPE_SPLIT, K_GEMM_O,
   K_RESID_NORM, K_GEMM_GATE_UP, K_SWIGLU, K_GEMM_DOWN, K_GEMM_F32, K_RESID_ADD, K_KERNEL_ID_END
 };
@@ -69,6 +69,7 @@ struct cascade_ctx {
   int attn_max_splits = 1;
   float* attn_part_o = nullptr;   // [R*Hq*splits][T_pad][D]
   float2* attn_part_ml = nullptr;  // [R*Hq*splits][T_pad]  (row max, row sum)
+  unsigned int* attn_unit_done = nullptr;  // [R*Hq*row blocks] finished-split counters (zero between launches)
 
   // LM head
   int head_m_pad = 0;             // B*T_max rounded up to 128
