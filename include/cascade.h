@@ -292,6 +292,37 @@ int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const c
                              uint8_t* accept_host, int32_t* path_nodes_host, int32_t* path_len_host,
                              void* stream);
 
+/* ---- acceptance without any device allocation --------------------------------------------------- */
+/* The paper has no counterpart to this entry point; it exists for deployment.  Some callers of this
+ * library may not allocate device memory at all: a plug-in running inside a serving process that
+ * handed its whole memory budget to one arena at start-up, code that runs after the host has frozen
+ * allocation (for instance to keep addresses stable), or a process whose allocator hooks forbid
+ * cudaMalloc.  cascade_create and cascade_tree_create call cudaMalloc, so such callers cannot use the
+ * entry points above.  This one needs neither object: similarity scores (Section 4.1), relaxed acceptance
+ * (Eq. 1-3, Algorithm 2) and path selection, as cascade_similarity + cascade_relaxed_accept +
+ * cascade_select_path compute them, with all device-side scratch (the tree descriptor, the cosine
+ * scores, the per-prompt finished-CTA counters) in one static device array of the library
+ * (about 0.7 MB, held by every GPU that loads the library until the process exits).
+ *   B <= CASCADE_STATIC_MAX_PROMPTS, T <= CASCADE_MAX_TREE_ROWS; larger sizes return
+ *   CASCADE_ERR_UNSUPPORTED_SHAPE and nothing is launched.
+ *   parent [T]: HOST array, same rules as cascade_tree_create.  Everything else: device pointers with the
+ *   meaning they have in cascade_similarity / cascade_relaxed_accept / cascade_select_path
+ *   (feat [B,T,feat_dim] float, 16-byte aligned; feat_norm [B,T] or NULL; row_lse, cand_parent,
+ *   cand_gparent [B,T]; tok, draft_p, uniforms [B,T]; outputs accept [B,T], path_nodes [B,depth+1],
+ *   path_len [B]; q_relaxed, tvd_out, near_count, tvd_used may be NULL).
+ * The call allocates nothing on the device: it copies the tree descriptor into the static array, clears
+ * the counters and enqueues one kernel on `stream`.  The first call on a device also looks up the device
+ * address of the array (cudaGetSymbolAddress), so make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the last call's contents: two calls whose
+ * work overlaps on the GPU (different streams) race; serialise them. */
+#define CASCADE_STATIC_MAX_PROMPTS 32
+int cascade_accept_static(int32_t B, int32_t T, const int32_t* parent, const float* feat, int32_t feat_dim,
+                          const float* feat_norm, const float* row_lse, const float* cand_parent,
+                          const float* cand_gparent, const int32_t* tok, const float* draft_p,
+                          const float* uniforms, const cascade_params* params, int32_t select_mode,
+                          uint8_t* accept, float* q_relaxed, float* tvd_out, int32_t* near_count,
+                          int32_t* path_nodes, int32_t* path_len, float* tvd_used, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

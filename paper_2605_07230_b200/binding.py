@@ -27,7 +27,7 @@ EXPORTS = [
     "cascade_strerror", "cascade_timing_enable", "cascade_timing_read", "cascade_kernel_name", "cascade_tree_create", "cascade_tree_destroy", "cascade_tree_rows", "cascade_tree_depth",
     "cascade_tree_num_pairs", "cascade_tree_pairs", "cascade_tree_attn", "cascade_lm_head_cfg",
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
-    "cascade_verify_step_host",
+    "cascade_verify_step_host", "cascade_accept_static",
 ]
 
 
@@ -97,6 +97,8 @@ def lib() -> C.CDLL:
         L.cascade_select_path.argtypes = [vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
         L.cascade_verify_step.argtypes = [vp, vp, C.POINTER(Step), vp]
         L.cascade_verify_step_host.argtypes = [vp, vp, C.POINTER(Step), vp, vp, vp, vp, vp, vp, vp]
+        L.cascade_accept_static.argtypes = [C.c_int32, C.c_int32, vp, vp, C.c_int32, vp, vp, vp, vp, vp, vp, vp,
+                                            C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -277,3 +279,16 @@ def cascade_verify_step_host(ctx, tree, step: Step, tok_host, draft_p_host, unif
     _check(lib().cascade_verify_step_host(ctx.handle, tree.handle, C.byref(step), _ptr(tok_host),
                                           _ptr(draft_p_host), _ptr(uniforms_host), _ptr(accept_host),
                                           _ptr(path_nodes_host), _ptr(path_len_host), _stream()))
+
+
+def cascade_accept_static(B, parent, feat, feat_dim, feat_norm, row_lse, cand_parent, cand_gparent, tok, draft_p,
+                          uniforms, params: Params, select_mode, accept, q_relaxed, tvd_out, near_count, path_nodes,
+                          path_len, tvd_used):
+    """Scores + relaxed acceptance + path selection with no context, no tree object and no device
+    allocation (the library's static device array is the only scratch).  `parent` is a host sequence."""
+    arr = (C.c_int32 * len(parent))(*[int(x) for x in parent])
+    _check(lib().cascade_accept_static(B, len(parent), arr, _ptr(feat), feat_dim, _ptr(feat_norm), _ptr(row_lse),
+                                       _ptr(cand_parent), _ptr(cand_gparent), _ptr(tok), _ptr(draft_p),
+                                       _ptr(uniforms), C.byref(params), select_mode, _ptr(accept), _ptr(q_relaxed),
+                                       _ptr(tvd_out), _ptr(near_count), _ptr(path_nodes), _ptr(path_len),
+                                       _ptr(tvd_used), _stream()))
