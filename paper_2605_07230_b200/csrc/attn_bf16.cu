@@ -35,6 +35,7 @@ constexpr int kPBytes = 128 * kTileKeys * 2;  // 32 KB
 constexpr int kKVTileBytes = kTileKeys * kD * 2;  // 32 KB for K, same for V
 constexpr int kStageBytes = 2 * kKVTileBytes;
 constexpr int kStages = 2;
+constexpr int kPrefetch = 6;  // K/V tiles requested into the L2 ahead of the shared-memory ring
 constexpr int kSmemBytes = kQBytes + kPBytes + kStages * kStageBytes + 1024;
 constexpr int kXRow = 133;  // row stride (floats) of the half-merge exchange buffer
 
@@ -119,9 +120,24 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int copy = 0; copy < 2; ++copy)
           ptx::tma_load_4d(smem + half * (kQBytes / 2) + copy * (64 * 128), &tm_q, half * 64, head,
                            rb * kRowsPerBlock, r, &q_full);
+      // The ring holds two tiles, which is less than the HBM latency x this SM's share of the bandwidth:
+      // tiles further ahead are pulled into the L2 so that the ring is refilled at L2 latency.
+      auto prefetch = [&](int i) {
+        const int tile = tile_begin + i;
+        const bool in_prefix = tile < n_ptiles;
+        const CUtensorMap* mk = in_prefix ? &tm_kp : &tm_kt;
+        const CUtensorMap* mv = in_prefix ? &tm_vp : &tm_vt;
+        const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys;
+        for (int half = 0; half < 2; ++half) {
+          ptx::tma_prefetch_4d(mk, half * 64, hk, key0, r);
+          ptx::tma_prefetch_4d(mv, half * 64, hk, key0, r);
+        }
+      };
+      for (int i = kStages; i < min(n, kStages + kPrefetch); ++i) prefetch(i);
       for (int i = 0; i < n; ++i) {
         const int s = i % kStages;
         const uint32_t ph = (i / kStages) & 1u;
+        if (i + kStages + kPrefetch < n) prefetch(i + kStages + kPrefetch);
         if (!ptx::mbar_wait(&kv_empty[s], ph ^ 1u, abort_flag, p.err)) break;
         const int tile = tile_begin + i;
         const bool in_prefix = tile < n_ptiles;
