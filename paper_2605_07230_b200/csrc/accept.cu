@@ -191,30 +191,47 @@ __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
   for (int d = 0; d < tr.depth_max; ++d) {
     if (j < T && s_depth[j] == d && s_cc[j] > 0) {
       float t = s_tvd[j];
-      const int cb = s_cb[j], ce = cb + s_cc[j];
-      for (int i = cb; i < ce; ++i) {
-        float qR = s_q[i];
-        uint8_t near = 0;
-        const uint8_t has = s_has[i];
-        if (has & 1) {
-          const float m = s_mI[i];
-          if (fabsf(t + m - prm.tvd_budget) < CASCADE_NEAR) near |= 2;
-          if (t + m <= prm.tvd_budget) {
-            qR += m;
-            t += m;
+      const int cb = s_cb[j], cc = s_cc[j];
+      // four children at a time: their data is read first (independent shared-memory loads), the
+      // running total then moves through registers only
+      for (int base = 0; base < cc; base += 4) {
+        float q4[4], mI4[4], mC4[4];
+        uint32_t has4[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = cb + min(base + u, cc - 1);
+          q4[u] = s_q[i];
+          mI4[u] = s_mI[i];
+          mC4[u] = s_mC[i];
+          has4[u] = s_has[i];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (base + u < cc) {
+            const int i = cb + base + u;
+            float qR = q4[u];
+            uint32_t near = 0;
+            if (has4[u] & 1u) {
+              const float m = mI4[u];
+              if (fabsf(t + m - prm.tvd_budget) < CASCADE_NEAR) near |= 2;
+              if (t + m <= prm.tvd_budget) {
+                qR += m;
+                t += m;
+              }
+            }
+            if (has4[u] & 2u) {
+              const float m = mC4[u];
+              if (fabsf(t + m - prm.tvd_budget) < CASCADE_NEAR) near |= 2;
+              if (t + m <= prm.tvd_budget) {
+                qR += m;
+                t += m;
+              }
+            }
+            s_tvd[i] = t;
+            s_qR[i] = qR;
+            if (near) s_near[i] |= (uint8_t)near;
           }
         }
-        if (has & 2) {
-          const float m = s_mC[i];
-          if (fabsf(t + m - prm.tvd_budget) < CASCADE_NEAR) near |= 2;
-          if (t + m <= prm.tvd_budget) {
-            qR += m;
-            t += m;
-          }
-        }
-        s_tvd[i] = t;
-        s_qR[i] = qR;
-        s_near[i] |= near;
       }
     }
     __syncthreads();

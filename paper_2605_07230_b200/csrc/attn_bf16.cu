@@ -4,7 +4,8 @@
 // (CFG row, head) and shared by all tree rows.
 //
 // One CTA per (KV split, query head x row block, CFG row):
-//   * a TMA producer warp streams 128-key K and V tiles (bf16, 128-byte swizzle) through a 2-stage ring;
+//   * two producer threads stream 128-key K tiles and V tiles (bf16, 128-byte swizzle) through their own
+//     rings (2 and 3 slots) and ask the L2 for the tiles after those;
 //   * one thread issues the tensor-core work: S = Q K^T (UMMA 128x128x128) into one of two TMEM score
 //     buffers, and O_tile = P V into one of two TMEM output buffers;
 //   * four softmax warps own the 128 TMEM lanes.  A row block holds at most 64 tree rows, and the
@@ -33,10 +34,10 @@ constexpr int kThreads = 192;  // warps 0-3 softmax, warp 4 TMA, warp 5 UMMA iss
 constexpr int kQBytes = 128 * kD * 2;        // 32 KB: two 64-wide halves of [128 rows][64] bf16
 constexpr int kPBytes = 128 * kTileKeys * 2;  // 32 KB
 constexpr int kKVTileBytes = kTileKeys * kD * 2;  // 32 KB for K, same for V
-constexpr int kStageBytes = 2 * kKVTileBytes;
-constexpr int kStages = 2;
-constexpr int kPrefetch = 6;  // K/V tiles requested into the L2 ahead of the shared-memory ring
-constexpr int kSmemBytes = kQBytes + kPBytes + kStages * kStageBytes + 1024;
+constexpr int kKSlots = 2;     // K tiles in shared memory (a slot is free again once S = Q K^T has read it)
+constexpr int kVSlots = 3;     // V tiles in shared memory (free once O += P V has read it)
+constexpr int kPrefetch = 2;   // tiles requested into the L2 beyond what the shared-memory rings hold
+constexpr int kSmemBytes = kQBytes + kPBytes + (kKSlots + kVSlots) * kKVTileBytes + 1024;
 constexpr int kXRow = 133;  // row stride (floats) of the half-merge exchange buffer
 
 struct AttnArgs {
@@ -56,15 +57,16 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                  const __grid_constant__ CUtensorMap tm_vp, const __grid_constant__ CUtensorMap tm_kt,
                  const __grid_constant__ CUtensorMap tm_vt, const AttnArgs p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t q_full, kv_full[kStages], kv_empty[kStages], s_full[2], s_empty[2], p_full,
-      o_full[2], o_empty[2];
+  __shared__ __align__(8) uint64_t q_full, k_full[kKSlots], k_empty[kKSlots], v_full[kVSlots], v_empty[kVSlots],
+      s_full[2], s_empty[2], p_full, o_full;
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort, s_last;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const uint32_t q_addr = smem_base, p_addr = smem_base + kQBytes, kv_addr = p_addr + kPBytes;
+  const uint32_t q_addr = smem_base, p_addr = smem_base + kQBytes, k_ring = p_addr + kPBytes,
+                 v_ring = k_ring + kKSlots * kKVTileBytes;
 
   const int split = blockIdx.x, head = blockIdx.y / p.n_rb, rb = blockIdx.y % p.n_rb, r = blockIdx.z;
   const int hk = head / (p.Hq / p.Hkv);
@@ -79,33 +81,39 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(&q_full, 1);
-    for (int i = 0; i < kStages; ++i) {
-      ptx::mbar_init(&kv_full[i], 1);
-      ptx::mbar_init(&kv_empty[i], 1);
+    for (int i = 0; i < kKSlots; ++i) {
+      ptx::mbar_init(&k_full[i], 1);
+      ptx::mbar_init(&k_empty[i], 1);
+    }
+    for (int i = 0; i < kVSlots; ++i) {
+      ptx::mbar_init(&v_full[i], 1);
+      ptx::mbar_init(&v_empty[i], 1);
     }
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&s_full[i], 1);
       ptx::mbar_init(&s_empty[i], 128);
-      ptx::mbar_init(&o_full[i], 1);
-      ptx::mbar_init(&o_empty[i], 128);
     }
     ptx::mbar_init(&p_full, 128);
+    ptx::mbar_init(&o_full, 1);
     s_abort = 0;
     ptx::fence_mbar_init();
   }
-  // P starts at zero: each UMMA row only ever writes its own key half
-  for (int i = threadIdx.x; i < kPBytes / 16; i += kThreads)
-    reinterpret_cast<uint4*>(smem + kQBytes)[i] = make_uint4(0, 0, 0, 0);
-  ptx::fence_proxy_async_smem();
-  if (warp == 5) {
-    ptx::tmem_alloc(&s_tmem_base, 512);
-    ptx::tmem_relinquish();
-  }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::tc_fence_after();
-  const uint32_t tmem_base = s_tmem_base;
+  __syncthreads();  // barriers are initialised: the producers start streaming at once
   volatile int* abort_flag = &s_abort;
+  if (warp != 4) {
+    // meanwhile the other warps zero P (each UMMA row only ever writes its own key half) and get TMEM
+    for (int i = warp == 5 ? 128 + lane : threadIdx.x; i < kPBytes / 16; i += 160)
+      reinterpret_cast<uint4*>(smem + kQBytes)[i] = make_uint4(0, 0, 0, 0);
+    ptx::fence_proxy_async_smem();
+    if (warp == 5) {
+      ptx::tmem_alloc(&s_tmem_base, 512);
+      ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    ptx::named_bar_sync(2, 160);
+    ptx::tc_fence_after();
+  }
+  const uint32_t tmem_base = warp != 4 ? s_tmem_base : 0u;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
 
   // softmax state (warps 0-3)
@@ -113,85 +121,119 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   float m_run = -INFINITY, l_run = 0.f;
 
   if (warp == 4) {
-    // ---------------- TMA producer ----------------
-    if (lane == 0 && n > 0) {
-      ptx::mbar_arrive_expect_tx(&q_full, kQBytes);
-      for (int half = 0; half < 2; ++half)
-        for (int copy = 0; copy < 2; ++copy)
-          ptx::tma_load_4d(smem + half * (kQBytes / 2) + copy * (64 * 128), &tm_q, half * 64, head,
-                           rb * kRowsPerBlock, r, &q_full);
-      // The ring holds two tiles, which is less than the HBM latency x this SM's share of the bandwidth:
-      // tiles further ahead are pulled into the L2 so that the ring is refilled at L2 latency.
-      auto prefetch = [&](int i) {
-        const int tile = tile_begin + i;
-        const bool in_prefix = tile < n_ptiles;
-        const CUtensorMap* mk = in_prefix ? &tm_kp : &tm_kt;
-        const CUtensorMap* mv = in_prefix ? &tm_vp : &tm_vt;
-        const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys;
-        for (int half = 0; half < 2; ++half) {
-          ptx::tma_prefetch_4d(mk, half * 64, hk, key0, r);
-          ptx::tma_prefetch_4d(mv, half * 64, hk, key0, r);
-        }
-      };
-      for (int i = kStages; i < min(n, kStages + kPrefetch); ++i) prefetch(i);
+    // ---------------- TMA producers: lane 0 streams Q and the K tiles, lane 1 the V tiles ----------------
+    // The rings hold less than HBM latency x this SM's share of the bandwidth, so tiles further ahead
+    // are also requested into the L2 (each request after the tile load it accompanies: the TMA unit works in order).
+    if (lane < 2 && n > 0) {
+      const bool is_v = lane == 1;
+      const int slots = is_v ? kVSlots : kKSlots;
+      uint64_t* full = is_v ? v_full : k_full;
+      uint64_t* empty = is_v ? v_empty : k_empty;
+      const uint32_t ring_off = (is_v ? v_ring : k_ring) - smem_base;
+      if (!is_v) {
+        ptx::mbar_arrive_expect_tx(&q_full, kQBytes);
+        for (int half = 0; half < 2; ++half)
+          for (int copy = 0; copy < 2; ++copy)
+            ptx::tma_load_4d(smem + half * (kQBytes / 2) + copy * (64 * 128), &tm_q, half * 64, head,
+                             rb * kRowsPerBlock, r, &q_full);
+      }
+      int slot = 0;
+      uint32_t ph = 0;
       for (int i = 0; i < n; ++i) {
-        const int s = i % kStages;
-        const uint32_t ph = (i / kStages) & 1u;
-        if (i + kStages + kPrefetch < n) prefetch(i + kStages + kPrefetch);
-        if (!ptx::mbar_wait(&kv_empty[s], ph ^ 1u, abort_flag, p.err)) break;
+        if (!ptx::mbar_wait(&empty[slot], ph ^ 1u, abort_flag, p.err)) break;
         const int tile = tile_begin + i;
         const bool in_prefix = tile < n_ptiles;
-        const CUtensorMap* mk = in_prefix ? &tm_kp : &tm_kt;
-        const CUtensorMap* mv = in_prefix ? &tm_vp : &tm_vt;
+        const CUtensorMap* m = is_v ? (in_prefix ? &tm_vp : &tm_vt) : (in_prefix ? &tm_kp : &tm_kt);
         const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys;
-        uint8_t* stage = smem + kQBytes + kPBytes + s * kStageBytes;
-        ptx::mbar_arrive_expect_tx(&kv_full[s], kStageBytes);
-        for (int half = 0; half < 2; ++half) {
-          ptx::tma_load_4d(stage + half * (kKVTileBytes / 2), mk, half * 64, hk, key0, r, &kv_full[s]);
-          ptx::tma_load_4d(stage + kKVTileBytes + half * (kKVTileBytes / 2), mv, half * 64, hk, key0, r,
-                           &kv_full[s]);
+        uint8_t* dst = smem + ring_off + slot * kKVTileBytes;
+        ptx::mbar_arrive_expect_tx(&full[slot], kKVTileBytes);
+        ptx::tma_load_4d(dst, m, 0, hk, key0, r, &full[slot]);
+        ptx::tma_load_4d(dst + kKVTileBytes / 2, m, 64, hk, key0, r, &full[slot]);
+        if (++slot == slots) {
+          slot = 0;
+          ph ^= 1u;
+        }
+        // and ask the L2 for the tile kPrefetch beyond the ring (one per tile: a burst of requests would
+        // queue in front of the loads the ring is waiting for)
+        const int t = i + slots + kPrefetch - 1;
+        if (t < n) {
+          const int tile2 = tile_begin + t;
+          const bool pre2 = tile2 < n_ptiles;
+          const CUtensorMap* m2 = is_v ? (pre2 ? &tm_vp : &tm_vt) : (pre2 ? &tm_kp : &tm_kt);
+          const int key2 = (pre2 ? tile2 : tile2 - n_ptiles) * kTileKeys;
+          ptx::tma_prefetch_4d(m2, 0, hk, key2, r);
+          ptx::tma_prefetch_4d(m2, 64, hk, key2, r);
         }
       }
     }
   } else if (warp == 5) {
     // ---------------- UMMA issue ----------------
+    // S(i) = Q K_i^T needs K tile i and a free score buffer; O += P_i V_i needs the softmax of tile i and
+    // V tile i.  Whichever is ready is issued, so scores run ahead of the softmax while the output product
+    // never waits for the next tile's keys.
     if (lane == 0 && n > 0) {
       const uint32_t idesc_s = ptx::umma_idesc_bf16(128, kTileKeys);
       const uint32_t idesc_o = ptx::umma_idesc_bf16_b_mn(128, kD);
-      auto issue_s = [&](int i) -> bool {
-        const int s = i % kStages;
-        if (!ptx::mbar_wait(&kv_full[s], (i / kStages) & 1u, abort_flag, p.err)) return false;
-        if (!ptx::mbar_wait(&s_empty[i & 1], ((i >> 1) & 1u) ^ 1u, abort_flag, p.err)) return false;
-        ptx::tc_fence_after();
-        const uint32_t k_addr = kv_addr + s * kStageBytes;
-#pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
-          ptx::umma_bf16(tmem_s + (i & 1) * 128, ptx::umma_desc_sw128(q_addr + off),
-                         ptx::umma_desc_sw128(k_addr + off), idesc_s, ks != 0);
-        }
-        ptx::umma_commit(&s_full[i & 1]);
-        return true;
-      };
       bool ok = ptx::mbar_wait(&q_full, 0, abort_flag, p.err);
-      ok = ok && issue_s(0);
-      for (int i = 0; ok && i < n; ++i) {
-        if (i + 1 < n && !issue_s(i + 1)) break;
-        if (!ptx::mbar_wait(&p_full, i & 1u, abort_flag, p.err)) break;
-        if (!ptx::mbar_wait(&o_empty[i & 1], ((i >> 1) & 1u) ^ 1u, abort_flag, p.err)) break;
-        ptx::tc_fence_after();
-        const uint32_t v_addr = kv_addr + (i % kStages) * kStageBytes + kKVTileBytes;
+      int is = 0, ip = 0;             // next S, next PV
+      int ks_slot = 0, vs_slot = 0;   // ring positions
+      uint32_t k_ph = 0, v_ph = 0;
+      uint64_t t_idle = 0;
+      uint32_t polls = 0;
+      while (ok && ip < n) {
+        bool did = false;
+        if (is < n && ptx::mbar_test_wait(&k_full[ks_slot], k_ph) &&
+            ptx::mbar_test_wait(&s_empty[is & 1], ((is >> 1) & 1u) ^ 1u)) {
+          ptx::tc_fence_after();
+          const uint32_t k_addr = k_ring + ks_slot * kKVTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < kTileKeys / 16; ++ks) {
-          // A = P: K-major, two 64-key column blocks of [128 rows][128 B]
-          const uint64_t pd = ptx::umma_desc_sw128(p_addr + (ks >> 2) * (128 * 128) + (ks & 3) * 32);
-          // B = V: [key][d] with d contiguous (MN-major); 16 keys = two 8-row groups of 1 KB;
-          // the two 64-wide halves of d are 16 KB apart
-          const uint64_t vd = ptx::umma_desc_sw128_strides(v_addr + ks * 2048, kKVTileBytes / 2, 1024);
-          ptx::umma_bf16(tmem_o + (i & 1) * 128, pd, vd, idesc_o, ks != 0);
+          for (int ks = 0; ks < kD / 16; ++ks) {
+            const uint32_t off = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
+            ptx::umma_bf16(tmem_s + (is & 1) * 128, ptx::umma_desc_sw128(q_addr + off),
+                           ptx::umma_desc_sw128(k_addr + off), idesc_s, ks != 0);
+          }
+          ptx::umma_commit(&s_full[is & 1]);
+          ptx::umma_commit(&k_empty[ks_slot]);
+          if (++ks_slot == kKSlots) {
+            ks_slot = 0;
+            k_ph ^= 1u;
+          }
+          ++is;
+          did = true;
         }
-        ptx::umma_commit(&o_full[i & 1]);
-        ptx::umma_commit(&kv_empty[i % kStages]);
+        if (ip < is && ptx::mbar_test_wait(&p_full, ip & 1u) && ptx::mbar_test_wait(&v_full[vs_slot], v_ph)) {
+          ptx::tc_fence_after();
+          const uint32_t v_addr = v_ring + vs_slot * kKVTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < kTileKeys / 16; ++ks) {
+            // A = P: K-major, two 64-key column blocks of [128 rows][128 B]
+            const uint64_t pd = ptx::umma_desc_sw128(p_addr + (ks >> 2) * (128 * 128) + (ks & 3) * 32);
+            // B = V: [key][d] with d contiguous (MN-major); 16 keys = two 8-row groups of 1 KB;
+            // the two 64-wide halves of d are 16 KB apart
+            const uint64_t vd = ptx::umma_desc_sw128_strides(v_addr + ks * 2048, kKVTileBytes / 2, 1024);
+            ptx::umma_bf16(tmem_o, pd, vd, idesc_o, (ip | ks) != 0);  // O accumulates across tiles
+          }
+          ptx::umma_commit(&o_full);
+          ptx::umma_commit(&v_empty[vs_slot]);
+          if (++vs_slot == kVSlots) {
+            vs_slot = 0;
+            v_ph ^= 1u;
+          }
+          ++ip;
+          did = true;
+        }
+        if (did) {
+          polls = 0;
+        } else if ((++polls & 255u) == 0) {  // bounded: give up after the wait limit without progress
+          if (*abort_flag) break;
+          const uint64_t now = ptx::global_timer_ns();
+          if (polls == 256u) t_idle = now;
+          if (now - t_idle > ptx::kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicOr(p.err, 1);
+            break;
+          }
+        }
       }
     }
   } else {
@@ -201,15 +243,18 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int khalf = urow >> 6;              // which 64 keys of each tile this lane owns
     const int j = rb * kRowsPerBlock + row_in_block;  // tree row
     const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-#pragma unroll
-    for (int d = 0; d < kD; ++d) o_acc[d] = 0.f;
-    float alpha_prev = 1.f;
     uint64_t anc_w[4] = {0, 0, 0, 0};
     if (j < p.T) {
 #pragma unroll
       for (int w = 0; w < 4; ++w) anc_w[w] = p.anc[(size_t)j * 4 + w];
     }
     const uint32_t p_row_addr = p_addr + khalf * (128 * 128) + urow * 128;
+    const uint32_t o_addr = tmem_o + lane_addr;
+    // Online softmax with a lazily updated reference: weights are 2^(s - m_run) where m_run is only
+    // raised when a tile's maximum exceeds it by more than kLazy (so weights stay below 2^kLazy).
+    // The outputs then accumulate across tiles inside TMEM (the UMMA adds into O); this lane's O and
+    // sum are rescaled only on the rare tile that raises m_run.
+    constexpr float kLazy = 8.f;
     bool ok = n > 0;
     for (int i = 0; ok && i < n; ++i) {
       if (!ptx::mbar_wait(&s_full[i & 1], (i >> 1) & 1u, abort_flag, p.err)) { ok = false; break; }
@@ -226,19 +271,23 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         vis = anc_w[(key0 >> 6) & 3];
       }
       float sc[64];
-      const uint32_t s_addr = tmem_s + lane_addr + (i & 1) * 128 + khalf * 64;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) ptx::tmem_ld16(s_addr + c * 16, sc + c * 16);
+      ptx::tmem_ld64(tmem_s + lane_addr + (i & 1) * 128 + khalf * 64, sc);
       ptx::tc_fence_before();
       ptx::mbar_arrive(&s_empty[i & 1]);
-      float m_new = m_run;
+      float m_tile = -INFINITY;
 #pragma unroll
       for (int k = 0; k < 64; ++k) {
         sc[k] = ((vis >> k) & 1ull) ? sc[k] * p.c : -INFINITY;
-        m_new = fmaxf(m_new, sc[k]);
+        m_tile = fmaxf(m_tile, sc[k]);
       }
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      const float alpha = m_run == -INFINITY ? 1.f : ptx::ex2(m_run - m_use);
+      float alpha = 1.f;  // factor for what this lane has accumulated so far
+      if (m_run == -INFINITY) {
+        m_run = m_tile;   // nothing accumulated yet (all weights so far were zero)
+      } else if (m_tile > m_run + kLazy) {
+        alpha = ptx::ex2(m_run - m_tile);
+        m_run = m_tile;
+      }
+      const float m_use = m_run == -INFINITY ? 0.f : m_run;
       float rowsum = 0.f;
       uint32_t packed[32];
 #pragma unroll
@@ -249,8 +298,20 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         rowsum += __uint_as_float(packed[k >> 1] << 16) + __uint_as_float(packed[k >> 1] & 0xffff0000u);
       }
       if (i >= 1) {
-        // PV(i-1) complete: P may be overwritten and O_{i-1} is ready
-        if (!ptx::mbar_wait(&o_full[(i - 1) & 1], ((i - 1) >> 1) & 1u, abort_flag, p.err)) { ok = false; break; }
+        // PV(i-1) complete: P may be overwritten and O holds tiles 0..i-1
+        if (!ptx::mbar_wait(&o_full, (i - 1) & 1u, abort_flag, p.err)) { ok = false; break; }
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+          ptx::tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            float t[16];
+            ptx::tmem_ld16(o_addr + c * 16, t);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) t[k] *= alpha;
+            ptx::tmem_st16(o_addr + c * 16, t);
+          }
+          ptx::tc_fence_before();
+        }
       }
 #pragma unroll
       for (int c = 0; c < 8; ++c)
@@ -258,40 +319,21 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                           packed[4 * c + 3]);
       ptx::fence_proxy_async_smem();
       ptx::mbar_arrive(&p_full);
-      if (i >= 1) {
-        ptx::tc_fence_after();
-        const uint32_t o_addr = tmem_o + lane_addr + ((i - 1) & 1) * 128;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          float t[16];
-          ptx::tmem_ld16(o_addr + c * 16, t);
-#pragma unroll
-          for (int k = 0; k < 16; ++k) o_acc[c * 16 + k] = o_acc[c * 16 + k] * alpha_prev + t[k];
-        }
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(&o_empty[(i - 1) & 1]);
-      }
       l_run = l_run * alpha + rowsum;
-      m_run = m_new;
-      alpha_prev = alpha;
     }
+#pragma unroll
+    for (int d = 0; d < kD; ++d) o_acc[d] = 0.f;
     if (ok && n > 0) {
-      if (ptx::mbar_wait(&o_full[(n - 1) & 1], ((n - 1) >> 1) & 1u, abort_flag, p.err)) {
+      if (ptx::mbar_wait(&o_full, (n - 1) & 1u, abort_flag, p.err)) {
         ptx::tc_fence_after();
-        const uint32_t o_addr = tmem_o + lane_addr + ((n - 1) & 1) * 128;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          float t[16];
-          ptx::tmem_ld16(o_addr + c * 16, t);
-#pragma unroll
-          for (int k = 0; k < 16; ++k) o_acc[c * 16 + k] = o_acc[c * 16 + k] * alpha_prev + t[k];
-        }
+        ptx::tmem_ld64(o_addr, o_acc);
+        ptx::tmem_ld64(o_addr + 64, o_acc + 64);
         ptx::tc_fence_before();
       }
     }
     // ---- merge the two key halves of each row (lanes r and r+64), then write ----
     // all UMMAs and TMA copies of this CTA have completed: the KV ring is free to reuse
-    float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);
+    float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);  // the K ring: 64 rows x 133 floats fit
     ptx::named_bar_sync(1, 128);
     if (khalf == 1) {
       float* x = xbuf + row_in_block * kXRow;
@@ -357,25 +399,41 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int row = threadIdx.x & 63, j = rb * kRowsPerBlock + row, d0 = (threadIdx.x >> 6) * (kD / 2);
   if (j >= p.T) return;
   const size_t unit0 = ((size_t)r * p.Hq + head) * p.splits;
+  // two splits per round, every load of a round issued before the first use
   float m = -INFINITY;
   for (int s = 0; s < p.splits; ++s) m = fmaxf(m, __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + j]).x);
   float acc[kD / 2];
 #pragma unroll
   for (int d = 0; d < kD / 2; ++d) acc[d] = 0.f;
   float l = 0.f;
-  for (int s = 0; s < p.splits; ++s) {
-    const float2 ml = __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + j]);
-    if (ml.x == -INFINITY) continue;
-    const float w = ptx::ex2(ml.x - m);
-    l += w * ml.y;
-    const float4* src = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s) * p.t_pad + j) * kD + d0);
+  for (int s0 = 0; s0 < p.splits; s0 += 2) {
+    const int s1 = min(s0 + 1, p.splits - 1);
+    const float2 ml0 = __ldcg(&p.part_ml[(unit0 + s0) * p.t_pad + j]);
+    const float2 ml1 = __ldcg(&p.part_ml[(unit0 + s1) * p.t_pad + j]);
+    const float4* src0 = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s0) * p.t_pad + j) * kD + d0);
+    const float4* src1 = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s1) * p.t_pad + j) * kD + d0);
+    float4 t0[kD / 8], t1[kD / 8];
+#pragma unroll
+    for (int c = 0; c < kD / 8; ++c) t0[c] = __ldcg(src0 + c);
+#pragma unroll
+    for (int c = 0; c < kD / 8; ++c) t1[c] = __ldcg(src1 + c);
+    const float w0 = ml0.x == -INFINITY ? 0.f : ptx::ex2(ml0.x - m);
+    const float w1 = (s1 == s0 || ml1.x == -INFINITY) ? 0.f : ptx::ex2(ml1.x - m);
+    l += w0 * ml0.y;
+    l += w1 * ml1.y;
 #pragma unroll
     for (int c = 0; c < kD / 8; ++c) {
-      const float4 t = __ldcg(src + c);
-      acc[4 * c] += w * t.x;
-      acc[4 * c + 1] += w * t.y;
-      acc[4 * c + 2] += w * t.z;
-      acc[4 * c + 3] += w * t.w;
+      acc[4 * c] += w0 * t0[c].x;
+      acc[4 * c + 1] += w0 * t0[c].y;
+      acc[4 * c + 2] += w0 * t0[c].z;
+      acc[4 * c + 3] += w0 * t0[c].w;
+    }
+#pragma unroll
+    for (int c = 0; c < kD / 8; ++c) {
+      acc[4 * c] += w1 * t1[c].x;
+      acc[4 * c + 1] += w1 * t1[c].y;
+      acc[4 * c + 2] += w1 * t1[c].z;
+      acc[4 * c + 3] += w1 * t1[c].w;
     }
   }
   const float inv = 1.f / l;
@@ -419,6 +477,8 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   int splits = ctx->sm_count / units;
   if (splits > n_tiles) splits = n_tiles;
   if (splits > ctx->attn_max_splits) splits = ctx->attn_max_splits;
+  // merging splits costs a few microseconds of its own: not worth it for a handful of tiles
+  if (splits > 1 && n_tiles - cascade_detail::ceil_div(n_tiles, splits) < 4) splits = 1;
   if (splits < 1) splits = 1;
   a.splits = splits;
 
