@@ -70,7 +70,7 @@ typedef struct cascade_tree cascade_tree;
 
 /* Fixed sizes of a context.  Supported: D in {64,128}; Hq a multiple of Hkv; h a multiple of 64;
  * V a multiple of 8; T_max <= CASCADE_MAX_TREE_ROWS; B >= 1.  ffn may be 0 if no decoder layer is
- * run through cascade_verify_step (otherwise a multiple of 64). */
+ * run through cascade_verify_step (otherwise a multiple of 8). */
 typedef struct {
   int32_t dtype; /* CASCADE_F32 or CASCADE_BF16: element type of q/k/v, hidden states and weights */
   int32_t B;
@@ -218,7 +218,10 @@ int cascade_select_path(cascade_ctx* ctx, const cascade_tree* tree, const uint8_
 /* One pre-norm decoder layer (the workload's architecture; the paper treats the target as given):
  * a = RMSNorm(x, gamma_attn); q,k,v = a Wq^T, a Wk^T, a Wv^T; rotary (half-split pairing) at position
  * prefix_len[r] + depth[j]; tree attention; x += attn Wo^T; m = RMSNorm(x, gamma_mlp);
- * x += (silu(m Wg^T) * (m Wu^T)) Wd^T.  Matrices are [out_features, in_features] elem. */
+ * x += (silu(m Wg^T) * (m Wu^T)) Wd^T.  Matrices are [out_features, in_features] elem.  wq, wk, wv must be
+ * stacked in memory in this order (wk = wq + Hq*D*h elements, wv = wk + Hkv*D*h), and so must w_gate, w_up
+ * (w_up = w_gate + ffn*h): each group runs as one projection; CASCADE_ERR_UNSUPPORTED_SHAPE otherwise.
+ * The bf16 path needs D = 128. */
 typedef struct {
   const float* gamma_attn; /* [h] */
   const void* wq;          /* [Hq*D, h]  */

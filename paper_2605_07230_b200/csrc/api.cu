@@ -69,6 +69,38 @@ int64_t carve(cascade_ctx* c, char* base) {
   cv.take(c->scores, (int64_t)s.B * c->max_pairs);
   cv.take(c->q_relaxed, BT);
   cv.take(c->tvd_out, BT);
+  if (s.ffn > 0) {
+    // decoder layers: residual stream, GEMM operands, per-slice projection outputs, rotated q/k/v
+    const int64_t RT = (int64_t)R * T;
+    const int64_t k_max = s.h > s.ffn ? s.h : s.ffn;
+    const int es = elem_size(s);
+    cv.take(c->x, RT * s.h);
+    if (s.dtype == CASCADE_BF16) {
+      c->act_lo_offset = align_up(RT * k_max, 128);
+      cv.take(c->act_hi, 2 * c->act_lo_offset);
+    } else {
+      cv.take(c->act_f32, RT * k_max);
+    }
+    int64_t need = 0;
+    const int shapes[4][2] = {{(s.Hq + 2 * s.Hkv) * s.D, s.h}, {s.h, s.Hq * s.D}, {2 * s.ffn, s.h}, {s.h, s.ffn}};
+    for (const auto& nk : shapes) {
+      const int S = s.dtype == CASCADE_BF16 ? gemm_tc_pick_splits(c->sm_count, (int)RT, nk[0], nk[1], c->layer_max_splits) : 1;
+      const int64_t f = (int64_t)S * RT * nk[0];
+      if (f > need) need = f;
+    }
+    c->gemm_out_floats = need;
+    cv.take(c->gemm_out, need);
+    char* p = nullptr;
+    cv.take(p, RT * s.Hq * s.D * es);
+    c->q_rot = p;
+    cv.take(p, RT * s.Hkv * s.D * es);
+    c->k_rot = p;
+    cv.take(p, RT * s.Hkv * s.D * es);
+    c->v_rot = p;
+    c->attn_lo_offset = s.dtype == CASCADE_BF16 ? align_up(RT * s.Hq * s.D, 128) : 0;
+    cv.take(p, (RT * s.Hq * s.D + c->attn_lo_offset) * es);
+    c->attn_out = p;
+  }
   cv.take(c->st_tok, BT);
   cv.take(c->st_draft_p, BT);
   cv.take(c->st_uniforms, BT);
@@ -87,7 +119,7 @@ int validate_shape(const cascade_shape* s) {
   if (s->T_max > CASCADE_MAX_TREE_ROWS) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (s->D != 64 && s->D != 128) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (s->Hq % s->Hkv != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
-  if (s->h % 64 != 0 || s->V % 8 != 0 || s->ffn % 64 != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (s->h % 64 != 0 || s->V % 8 != 0 || s->ffn % 8 != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if ((int64_t)s->B * s->T_max > (1 << 20)) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   return CASCADE_OK;
 }
@@ -341,7 +373,7 @@ static int tree_attn_impl(cascade_ctx* ctx, const cascade_tree* tree, const void
     return launch_tree_attn_bf16(ctx, tree, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_prefix,
                                  (const __nv_bfloat16*)v_prefix, prefix_cap, prefix_len,
                                  (const __nv_bfloat16*)k_tree, (const __nv_bfloat16*)v_tree, (__nv_bfloat16*)out,
-                                 softmax_scale, s);
+                                 nullptr, softmax_scale, s);
   return launch_tree_attn_f32(ctx, tree, (const float*)q, (const float*)k_prefix, (const float*)v_prefix,
                               prefix_cap, prefix_len, (const float*)k_tree, (const float*)v_tree, (float*)out,
                               softmax_scale, s);
@@ -362,7 +394,8 @@ int cascade_tree_attn(cascade_ctx* ctx, const cascade_tree* tree, const void* q,
 static int lm_head_impl(cascade_ctx* ctx, const cascade_tree* tree, const void* hidden, const float* rms_gamma,
                         float eps, const void* w_head, float cfg_scale, float temperature, const int32_t* tok,
                         float* logits_out, float* feat_out, float* feat_norm_out, float* row_lse_out,
-                        float* cand_parent_out, float* cand_gparent_out, bool fold_lse, cudaStream_t s) {
+                        float* cand_parent_out, float* cand_gparent_out, bool fold_lse, bool hidden_f32,
+                        cudaStream_t s) {
   if (ctx == nullptr || tree == nullptr || hidden == nullptr || rms_gamma == nullptr || w_head == nullptr)
     return CASCADE_ERR_INVALID_ARG;
   if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
@@ -372,7 +405,7 @@ static int lm_head_impl(cascade_ctx* ctx, const cascade_tree* tree, const void* 
       !aligned16(rms_gamma))
     return CASCADE_ERR_INVALID_ARG;
   if (row_lse_out == nullptr) row_lse_out = ctx->row_lse;
-  CASCADE_TRY(launch_final_norm_mix(ctx, tree->T, hidden, rms_gamma, eps, cfg_scale, 1.f / temperature, feat_out,
+  CASCADE_TRY(launch_final_norm_mix(ctx, tree->T, hidden, hidden_f32, rms_gamma, eps, cfg_scale, 1.f / temperature, feat_out,
                                     feat_norm_out, tok ? cand_parent_out : nullptr, tok ? cand_gparent_out : nullptr,
                                     s));
   if (ctx->shape.dtype == CASCADE_BF16) {
@@ -398,7 +431,7 @@ int cascade_lm_head_cfg(cascade_ctx* ctx, const cascade_tree* tree, const void* 
                         float* cand_parent_out, float* cand_gparent_out, void* stream) {
   if (ctx != nullptr) ctx->launches = 0;
   return lm_head_impl(ctx, tree, hidden, rms_gamma, eps, w_head, cfg_scale, temperature, tok, logits_out, feat_out,
-                      feat_norm_out, row_lse_out, cand_parent_out, cand_gparent_out, true, as_stream(stream));
+                      feat_norm_out, row_lse_out, cand_parent_out, cand_gparent_out, true, false, as_stream(stream));
 }
 
 // ---- (c) ------------------------------------------------------------------------------------------------
@@ -489,18 +522,22 @@ static int verify_step_impl(cascade_ctx* ctx, const cascade_tree* tree, const ca
   if (st->select_mode != CASCADE_SELECT_LONGEST && st->select_mode != CASCADE_SELECT_FIRST_ACCEPT)
     return CASCADE_ERR_INVALID_ARG;
   if (st->n_layers < 0) return CASCADE_ERR_INVALID_ARG;
-  if (st->n_layers > 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;  // decoder layers: not built yet
-  if (st->hidden_in == nullptr) return CASCADE_ERR_INVALID_ARG;
+  if (st->n_layers == 0 && st->hidden_in == nullptr) return CASCADE_ERR_INVALID_ARG;
   ctx->launches = 0;
-  if (st->q != nullptr)
+  const void* hidden = st->hidden_in;
+  if (st->n_layers > 0) {
+    CASCADE_TRY(run_layers(ctx, tree, st, s));
+    hidden = ctx->x;
+  } else if (st->q != nullptr) {
     CASCADE_TRY(tree_attn_impl(ctx, tree, st->q, st->k_prefix, st->v_prefix, st->prefix_cap, st->prefix_len,
                                st->k_tree, st->v_tree, st->attn_out, st->softmax_scale, s));
+  }
   float* feat = st->feat ? st->feat : ctx->feat;
   float* row_lse = st->row_lse ? st->row_lse : ctx->row_lse;
   const bool bf16 = ctx->shape.dtype == CASCADE_BF16;
-  CASCADE_TRY(lm_head_impl(ctx, tree, st->hidden_in, st->gamma_final, st->eps, st->w_head, st->cfg_scale,
-                           st->temperature, st->tok, st->logits, feat, ctx->feat_norm, row_lse, ctx->cand_parent,
-                           ctx->cand_gparent, false, s));
+  CASCADE_TRY(lm_head_impl(ctx, tree, hidden, st->gamma_final, st->eps, st->w_head, st->cfg_scale, st->temperature,
+                           st->tok, st->logits, feat, ctx->feat_norm, row_lse, ctx->cand_parent, ctx->cand_gparent, false,
+                           st->n_layers > 0, s));
   // cosines, row log-sum-exp (bf16: folded from the head's partials), the rule and the path: one launch
   TailWork w;
   w.feat = feat;

@@ -93,15 +93,17 @@ struct cascade_ctx {
 
   // decoder layer activations (allocated when ffn > 0)
   float* x = nullptr;            // [R*T][h] residual stream, fp32
-  __nv_bfloat16* act_hi = nullptr;  // [rows_pad][max(h,ffn,Hq*D)] GEMM operand, high part
-  __nv_bfloat16* act_lo = nullptr;
-  float* act_f32 = nullptr;      // [R*T][max(h,ffn,Hq*D)] GEMM operand (fp32 path)
-  float* gemm_out = nullptr;     // [R*T][max((Hq+2Hkv)*D, 2*ffn)] fp32 GEMM result
+  __nv_bfloat16* act_hi = nullptr;  // [R*T][max(h,ffn)] GEMM operand, high part; the remainder part follows at
+  int64_t act_lo_offset = 0;        // act_hi + act_lo_offset (elements)
+  float* act_f32 = nullptr;      // [R*T][max(h,ffn)] GEMM operand (fp32 path)
+  float* gemm_out = nullptr;     // [slices][R*T][N] fp32 projection results, one matrix per K slice
+  int64_t gemm_out_floats = 0;
+  int layer_max_splits = 16;
   void* q_rot = nullptr;         // [R,T,Hq,D] elem
   void* k_rot = nullptr;         // [R,T,Hkv,D] elem
   void* v_rot = nullptr;
-  void* attn_out = nullptr;      // [R,T,Hq,D] elem
-  int rows_pad = 0;
+  void* attn_out = nullptr;      // [R,T,Hq,D] elem; bf16: followed by the rounding remainder, same shape
+  int64_t attn_lo_offset = 0;    // elements from attn_out to that remainder
 
   // staging for the host-buffer entry point
   int32_t* st_tok = nullptr;
@@ -201,11 +203,12 @@ int launch_tree_attn_f32(cascade_ctx* ctx, const cascade_tree* tree, const float
 int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* q,
                           const __nv_bfloat16* kp, const __nv_bfloat16* vp, int prefix_cap,
                           const int32_t* prefix_len, const __nv_bfloat16* kt, const __nv_bfloat16* vt,
-                          __nv_bfloat16* out, float scale, cudaStream_t s);
+                          __nv_bfloat16* out, __nv_bfloat16* out_lo, float scale, cudaStream_t s);
 
 // head.cu (norm + mix producers, fp32 head) / gemm_tc.cu (tcgen05 GEMM)
 // cand_parent / cand_gparent (may be null) are cleared here; the head fills the entries that exist.
-int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const float* gamma, float eps,
+// hidden_f32: the hidden states are fp32 whatever the context's element type (the residual stream).
+int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidden_f32, const float* gamma, float eps,
                           float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
                           float* cand_parent, float* cand_gparent, cudaStream_t s);
 int launch_head_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* w_head, const int32_t* tok,
@@ -214,3 +217,6 @@ int launch_head_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* w_h
 // The row log-sum-exp is folded from the partials by launch_tail.
 int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* w_head,
                      const int32_t* tok, float* logits, float* cand_parent, float* cand_gparent, cudaStream_t s);
+
+// layer.cu: the decoder layers of a verification step; leaves the residual stream in ctx->x.
+int run_layers(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, cudaStream_t s);

@@ -51,6 +51,7 @@ constexpr int kTileWBytes = kTileN * kSpan * 2;
 
 struct GemmArgs {
   int M, N, NB, n_mchunks, n_kb, stages, tmem_cols;
+  int has_lo;              // 0: the activation operand is exact in bf16 (no remainder part)
   int stash;               // 1: TMEM has room for a third accumulator set (partials of split tiles)
   long long units;         // n_tiles * n_kb
   int n_tiles;
@@ -135,7 +136,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const int a_span_bytes = 2 * p.NB * kSpan * 2;  // one span of the activations: hi block then lo block
+  const int a_span_bytes = (1 + p.has_lo) * p.NB * kSpan * 2;  // one span of the activations: hi block [, lo block]
   const int stage_bytes = kWBytes + kSpans * a_span_bytes;
 
   if (threadIdx.x == 0) {
@@ -228,7 +229,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
               for (int ks = 0; ks < kSpan / 16; ++ks) {
                 // advancing 16 K elements = 32 bytes = 2 descriptor units inside the swizzle span
                 ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + 2 * ks, idesc, (q | ks) == 0 ? accumulate : 1u);
-                ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
+                if (p.has_lo) ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
               }
             }
           }
@@ -471,14 +472,17 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 
 int64_t gemm_tc_scratch_floats(int sm_count) { return (int64_t)sm_count * 2 * 128 * kTileN; }
 
-int gemm_tc_pick_splits(int sm_count, int N, int K, int max_splits) {
-  const int n_tiles = cascade_detail::ceil_div(N, kTileN), n_kb = cascade_detail::ceil_div(K, kSpan);
+int gemm_tc_pick_splits(int sm_count, int M, int N, int K, int max_splits) {
+  const int n_tiles = cascade_detail::ceil_div(N, kTileN) * cascade_detail::ceil_div(M, 128);
+  const int n_kb = cascade_detail::ceil_div(K, kSpan);
   int best = 1;
   long long best_cost = -1;
-  for (int s = 1; s <= max_splits && s <= n_kb; ++s) {
-    // time ~ rounds x K blocks per item, plus a little per slice for writing and re-reading its matrix
+  // a stage may carry two 64-wide K spans, and every slice needs at least one stage
+  for (int s = 1; s <= max_splits && s <= cascade_detail::ceil_div(K, 2 * kSpan); ++s) {
+    // time ~ rounds x K blocks per item (8 cost units per K block of one round: 148 x 16 KB of weights),
+    // plus writing and re-reading one output matrix per slice at about the same rate
     const long long rounds = cascade_detail::ceil_div(n_tiles * s, sm_count);
-    const long long cost = rounds * cascade_detail::ceil_div(n_kb, s) * 8 + s;
+    const long long cost = rounds * cascade_detail::ceil_div(n_kb, s) * 8 + (long long)s * M * N / 37500;
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
       best = s;
@@ -512,13 +516,15 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   // no faster on the stream and split the LM head of a 16384-token vocabulary over too few tiles.)
   const int halves = 1;
   const int budget = 227 * 1024 - 20 * 1024 - 1024;  // static shared + alignment slack
-  const int span_bytes = halves * kTileWBytes + 2 * a.NB * kSpan * 2;
+  a.has_lo = lo_offset != 0;
+  const int span_bytes = halves * kTileWBytes + (1 + a.has_lo) * a.NB * kSpan * 2;
   const int spans = budget / (2 * span_bytes) >= 3 ? 2 : 1;
   const int stage_bytes = spans * span_bytes;
   a.stages = budget / stage_bytes;
   if (a.stages > kMaxStages) a.stages = kMaxStages;
   if (a.stages < 2) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   a.n_kb = cascade_detail::ceil_div(K, kSpan * spans);
+  if (epi.splits > a.n_kb) return CASCADE_ERR_INVALID_ARG;  // a slice without a K block would have no result
   const int n_tiles = cascade_detail::ceil_div(N, halves * kTileN) * a.n_mchunks;
   a.units = (long long)n_tiles * a.n_kb;
   a.n_tiles = n_tiles;
@@ -529,9 +535,9 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   while (a.tmem_cols < (a.stash ? 3 : 2) * halves * a.NB) a.tmem_cols *= 2;
   const CUtensorMap* tw =
       get_tmap_2d_bf16(ctx, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(halves * kTileN), kSpan);
-  const uint64_t ad[3] = {(uint64_t)K, (uint64_t)M, 2};
-  const uint64_t as[2] = {(uint64_t)K, (uint64_t)lo_offset};
-  const uint32_t ab[3] = {kSpan, (uint32_t)a.NB, 2};
+  const uint64_t ad[3] = {(uint64_t)K, (uint64_t)M, a.has_lo ? 2u : 1u};
+  const uint64_t as[2] = {(uint64_t)K, a.has_lo ? (uint64_t)lo_offset : (uint64_t)K * M};
+  const uint32_t ab[3] = {kSpan, (uint32_t)a.NB, a.has_lo ? 2u : 1u};
   const CUtensorMap* ta = get_tmap_bf16(ctx, a_hi, 3, ad, as, ab);
   if (tw == nullptr || ta == nullptr) return CASCADE_ERR_CUDA;
   const int smem = a.stages * stage_bytes + 1024;

@@ -173,20 +173,24 @@ int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bflo
                         s);
 }
 
-int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, const float* gamma, float eps,
+int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidden_f32, const float* gamma, float eps,
                           float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
                           float* cand_parent, float* cand_gparent, cudaStream_t s) {
   const cascade_shape& sh = ctx->shape;
   dim3 grid(T, sh.B);
   KernelScope ks(ctx, K_FINAL_NORM_MIX, s);
-  if (sh.dtype == CASCADE_BF16)
-    k_final_norm_mix<__nv_bfloat16><<<grid, kNormThreads, 0, s>>>(
-        static_cast<const __nv_bfloat16*>(hidden), sh.B, T, sh.h, gamma, eps, cfg_scale, inv_temperature, feat,
-        feat_norm, ctx->head_a_hi, ctx->head_a_hi + ctx->head_lo_offset, nullptr, cand_parent, cand_gparent);
+  const bool bf16 = sh.dtype == CASCADE_BF16;
+  __nv_bfloat16* a_hi = bf16 ? ctx->head_a_hi : nullptr;
+  __nv_bfloat16* a_lo = bf16 ? ctx->head_a_hi + ctx->head_lo_offset : nullptr;
+  float* a_f32 = bf16 ? nullptr : ctx->head_a_f32;
+  if (bf16 && !hidden_f32)
+    k_final_norm_mix<__nv_bfloat16><<<grid, kNormThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(hidden), sh.B, T,
+                                                                  sh.h, gamma, eps, cfg_scale, inv_temperature, feat,
+                                                                  feat_norm, a_hi, a_lo, a_f32, cand_parent, cand_gparent);
   else
     k_final_norm_mix<float><<<grid, kNormThreads, 0, s>>>(static_cast<const float*>(hidden), sh.B, T, sh.h, gamma, eps,
-                                                          cfg_scale, inv_temperature, feat, feat_norm, nullptr,
-                                                          nullptr, ctx->head_a_f32, cand_parent, cand_gparent);
+                                                          cfg_scale, inv_temperature, feat, feat_norm, a_hi, a_lo, a_f32,
+                                                          cand_parent, cand_gparent);
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }

@@ -1,0 +1,274 @@
+// The decoder layer around the tree attention (support for the workloads that run the verification
+// step through a layer: the paper treats the target model as given, the architecture is the usual
+// pre-norm block with rotary embeddings and a SwiGLU MLP).
+//
+//     a = RMSNorm(x, gamma_attn);  q,k,v = a Wq^T, a Wk^T, a Wv^T;  rotary at prefix_len[r] + depth[j];
+//     tree attention;  x += attn Wo^T;  m = RMSNorm(x, gamma_mlp);  x += (silu(m Wg^T) * (m Wu^T)) Wd^T
+//
+// The projections run on the tensor-core GEMM in sliced mode (K cut into S slices, one output matrix
+// per slice); the row-wise kernels here add the S matrices while they do their own work, so no GEMM
+// waits for another CTA.  The residual stream x stays fp32; GEMM operands are written as a bf16 high
+// part plus a bf16 remainder.
+#include "cascade_internal.h"
+#include "gemm_tc.h"
+
+namespace {
+
+constexpr int kRowThreads = 256;
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < kRowThreads / 32; ++i) t += red[i];
+  return t;
+}
+
+__device__ __forceinline__ float elem_to_float(const float* p, size_t i) { return p[i]; }
+__device__ __forceinline__ float elem_to_float(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
+
+// writes one operand value: bf16 high part + remainder, or fp32
+__device__ __forceinline__ void put_operand(__nv_bfloat16* hi, __nv_bfloat16* lo, float* f32, size_t i, float a) {
+  if (hi != nullptr) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(a);
+    hi[i] = h;
+    lo[i] = __float2bfloat16_rn(a - __bfloat162float(h));
+  } else {
+    f32[i] = a;
+  }
+}
+
+// One CTA per row m = r * T + j of the CFG pair.
+//   x[m] (+)= ...: embed != null: x[m] = embed[tok[b, j]]            (first layer)
+//                  else          x[m] += sum_s slices[s][m]          (output of the previous projection)
+//   operand[m] = RMSNorm(x[m], gamma)                                (skipped when gamma == null)
+template <typename E>
+__global__ void __launch_bounds__(kRowThreads) k_resid_norm(float* __restrict__ x, int B, int T, int h,
+                                                            const E* __restrict__ embed,
+                                                            const int32_t* __restrict__ tok,
+                                                            const float* __restrict__ slices, int n_slices,
+                                                            long long slice_stride, const float* __restrict__ gamma,
+                                                            float eps, __nv_bfloat16* __restrict__ a_hi,
+                                                            __nv_bfloat16* __restrict__ a_lo, float* __restrict__ a_f32,
+                                                            float* __restrict__ x_copy) {
+  __shared__ float red[kRowThreads / 32];
+  const int m = blockIdx.x;
+  const int r = m / T, j = m - r * T, b = r % B;
+  float* xr = x + (size_t)m * h;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < h; i += kRowThreads) {
+    float v;
+    if (embed != nullptr) {
+      v = elem_to_float(embed, (size_t)tok[(size_t)b * T + j] * h + i);
+    } else {
+      v = xr[i];
+      for (int s = 0; s < n_slices; ++s) v += slices[(size_t)s * slice_stride + (size_t)m * h + i];
+    }
+    xr[i] = v;
+    if (x_copy != nullptr) x_copy[(size_t)m * h + i] = v;
+    ss += v * v;
+  }
+  if (gamma == nullptr) return;
+  ss = block_sum(ss, red);
+  const float rs = rsqrtf(ss / h + eps);
+  for (int i = threadIdx.x; i < h; i += kRowThreads) put_operand(a_hi, a_lo, a_f32, (size_t)m * h + i, xr[i] * rs * gamma[i]);
+}
+
+// q, k, v = sum of the projection's slices; rotary embedding (half-split pairing: (x[i], x[i + D/2]) turned
+// by pos * base^(-2i/D)) on q and k at pos = prefix_len[r] + depth[j]; results in the attention's
+// element type.  grid (T, R), one thread per (head, pair index).
+template <typename E>
+__global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restrict__ slices, int n_slices,
+                                                            long long slice_stride, int T, int Hq, int Hkv, int D,
+                                                            const int32_t* __restrict__ prefix_len,
+                                                            const int32_t* __restrict__ depth, float rope_base,
+                                                            E* __restrict__ q, E* __restrict__ k, E* __restrict__ v) {
+  const int j = blockIdx.x, r = blockIdx.y;
+  const size_t m = (size_t)r * T + j;
+  const int n_cols = (Hq + 2 * Hkv) * D, half = D / 2;
+  const float pos = (float)(prefix_len[r] + depth[j]);
+  auto col = [&](int c) {
+    float a = 0.f;
+    for (int s = 0; s < n_slices; ++s) a += slices[(size_t)s * slice_stride + m * n_cols + c];
+    return a;
+  };
+  auto store = [](E* dst, size_t i, float val) {
+    if constexpr (sizeof(E) == 2) dst[i] = __float2bfloat16_rn(val);
+    else dst[i] = val;
+  };
+  // rotated pairs of q and k
+  for (int t = threadIdx.x; t < (Hq + Hkv) * half; t += kRowThreads) {
+    const int head = t / half, i = t - head * half;
+    const int c0 = head * D + i;  // q heads first, then k heads: same column order as the projection
+    const float x1 = col(c0), x2 = col(c0 + half);
+    const float inv_freq = powf(rope_base, -2.f * (float)i / (float)D);
+    float sn, cs;
+    sincosf(pos * inv_freq, &sn, &cs);
+    const float y1 = x1 * cs - x2 * sn, y2 = x2 * cs + x1 * sn;
+    if (head < Hq) {
+      const size_t o = (m * Hq + head) * D + i;
+      store(q, o, y1);
+      store(q, o + half, y2);
+    } else {
+      const size_t o = (m * Hkv + (head - Hq)) * D + i;
+      store(k, o, y1);
+      store(k, o + half, y2);
+    }
+  }
+  for (int t = threadIdx.x; t < Hkv * D; t += kRowThreads) store(v, m * Hkv * D + t, col((Hq + Hkv) * D + t));
+}
+
+// act = silu(gate) * up from the slices of the fused gate/up projection ([.., 2*ffn]: gate then up).
+__global__ void __launch_bounds__(kRowThreads) k_swiglu(const float* __restrict__ slices, int n_slices,
+                                                        long long slice_stride, int ffn,
+                                                        __nv_bfloat16* __restrict__ a_hi,
+                                                        __nv_bfloat16* __restrict__ a_lo, float* __restrict__ a_f32) {
+  const size_t m = blockIdx.y;
+  for (int i = blockIdx.x * kRowThreads + threadIdx.x; i < ffn; i += gridDim.x * kRowThreads) {
+    float g = 0.f, u = 0.f;
+    for (int s = 0; s < n_slices; ++s) {
+      const float* row = slices + (size_t)s * slice_stride + m * 2 * ffn;
+      g += row[i];
+      u += row[ffn + i];
+    }
+    put_operand(a_hi, a_lo, a_f32, m * ffn + i, g / (1.f + expf(-g)) * u);
+  }
+}
+
+// Plain fp32 projection for the fp32 workload: C[m][n] = sum_k A[m][k] W[n][k]; a warp per weight row.
+__global__ void __launch_bounds__(256) k_gemm_f32(const float* __restrict__ A, const float* __restrict__ W, int M,
+                                                  int N, int K, float* __restrict__ C) {
+  const int n = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (n >= N) return;
+  for (int mi = 0; mi < 8; ++mi) {
+    const int m = blockIdx.y * 8 + mi;
+    if (m >= M) break;
+    float acc = 0.f;
+    for (int k = lane; k < K; k += 32) acc += A[(size_t)m * K + k] * W[(size_t)n * K + k];
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) C[(size_t)m * N + n] = acc;
+  }
+}
+
+struct Projection {
+  int n_slices;
+  long long slice_stride;
+};
+
+// out slices = operand x W^T for one weight matrix (or several stacked in memory).
+int project(cascade_ctx* ctx, const void* W, int N, int K, int M, bool operand_is_attn, int kernel_id, Projection* pr,
+            cudaStream_t s) {
+  pr->slice_stride = (long long)M * N;
+  if (ctx->shape.dtype == CASCADE_BF16) {
+    const int S = gemm_tc_pick_splits(ctx->sm_count, M, N, K, ctx->layer_max_splits);
+    pr->n_slices = S;
+    GemmEpilogue e;
+    e.C = ctx->gemm_out;
+    e.ldc = N;
+    e.splits = S;
+    e.slice_stride = pr->slice_stride;
+    if ((long long)S * M * N > ctx->gemm_out_floats) return CASCADE_ERR_WORKSPACE;
+    if (operand_is_attn)  // the attention wrote its output as a bf16 high part plus remainder
+      return launch_gemm_tc(ctx, (const __nv_bfloat16*)W, N, K, (const __nv_bfloat16*)ctx->attn_out, ctx->attn_lo_offset, M,
+                            e, kernel_id, s);
+    return launch_gemm_tc(ctx, (const __nv_bfloat16*)W, N, K, ctx->act_hi, ctx->act_lo_offset, M, e, kernel_id, s);
+  }
+  pr->n_slices = 1;
+  dim3 grid(cascade_detail::ceil_div(N, 8), cascade_detail::ceil_div(M, 8));
+  {
+    KernelScope ks(ctx, K_GEMM_F32, s);
+    k_gemm_f32<<<grid, 256, 0, s>>>(operand_is_attn ? (const float*)ctx->attn_out : ctx->act_f32, (const float*)W, M, N, K,
+                                    ctx->gemm_out);
+  }
+  CASCADE_CUDA_TRY(cudaGetLastError());
+  return CASCADE_OK;
+}
+
+template <typename E>
+int resid_norm(cascade_ctx* ctx, int T, const void* embed, const int32_t* tok, const Projection* pr, const float* gamma,
+               float eps, float* x_copy, int kernel_id, cudaStream_t s) {
+  const cascade_shape& sh = ctx->shape;
+  const int M = 2 * sh.B * T;
+  const bool bf16 = sh.dtype == CASCADE_BF16;
+  KernelScope ks(ctx, kernel_id, s);
+  k_resid_norm<E><<<M, kRowThreads, 0, s>>>(ctx->x, sh.B, T, sh.h, (const E*)embed, tok, ctx->gemm_out,
+                                            pr ? pr->n_slices : 0, pr ? pr->slice_stride : 0, gamma, eps,
+                                            bf16 ? ctx->act_hi : nullptr, bf16 ? ctx->act_hi + ctx->act_lo_offset : nullptr,
+                                            bf16 ? nullptr : ctx->act_f32, x_copy);
+  CASCADE_CUDA_TRY(cudaGetLastError());
+  return CASCADE_OK;
+}
+
+template <typename E>
+int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, cudaStream_t s) {
+  const cascade_shape& sh = ctx->shape;
+  const int T = tree->T, R = 2 * sh.B, M = R * T;
+  const int qkv_cols = (sh.Hq + 2 * sh.Hkv) * sh.D;
+  Projection pr = {0, 0};
+  for (int li = 0; li < st->n_layers; ++li) {
+    const cascade_layer& L = st->layers[li];
+    if (L.gamma_attn == nullptr || L.wq == nullptr || L.wk == nullptr || L.wv == nullptr || L.wo == nullptr ||
+        L.gamma_mlp == nullptr || L.w_gate == nullptr || L.w_up == nullptr || L.w_down == nullptr)
+      return CASCADE_ERR_INVALID_ARG;
+    if (st->prefix_cap > 0 && (L.k_prefix == nullptr || L.v_prefix == nullptr)) return CASCADE_ERR_INVALID_ARG;
+    // input norm (first layer: from the token embeddings; later: after adding the previous MLP output)
+    CASCADE_TRY(resid_norm<E>(ctx, T, li == 0 ? st->embed : nullptr, st->tok, li == 0 ? nullptr : &pr, L.gamma_attn,
+                              st->eps, nullptr, li == 0 ? K_EMBED_NORM : K_RESID_NORM, s));
+    // q, k, v: one projection when the three matrices are stacked in memory, else three
+    const size_t es = sizeof(E);
+    const bool stacked = (const char*)L.wk == (const char*)L.wq + (size_t)sh.Hq * sh.D * sh.h * es &&
+                         (const char*)L.wv == (const char*)L.wk + (size_t)sh.Hkv * sh.D * sh.h * es;
+    if (!stacked) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+    CASCADE_TRY(project(ctx, L.wq, qkv_cols, sh.h, M, false, K_GEMM_QKV, &pr, s));
+    E* k_rot = st->k_tree_out ? (E*)st->k_tree_out + (size_t)li * M * sh.Hkv * sh.D : (E*)ctx->k_rot;
+    E* v_rot = st->v_tree_out ? (E*)st->v_tree_out + (size_t)li * M * sh.Hkv * sh.D : (E*)ctx->v_rot;
+    {
+      KernelScope ks(ctx, K_ROPE_SPLIT, s);
+      k_rope_split<E><<<dim3(T, R), kRowThreads, 0, s>>>(ctx->gemm_out, pr.n_slices, pr.slice_stride, T, sh.Hq, sh.Hkv,
+                                                         sh.D, st->prefix_len, tree->d_depth, st->rope_base,
+                                                         (E*)ctx->q_rot, k_rot, v_rot);
+    }
+    CASCADE_CUDA_TRY(cudaGetLastError());
+    if (sh.dtype == CASCADE_BF16)
+      CASCADE_TRY(launch_tree_attn_bf16(ctx, tree, (const __nv_bfloat16*)ctx->q_rot, (const __nv_bfloat16*)L.k_prefix,
+                                        (const __nv_bfloat16*)L.v_prefix, st->prefix_cap, st->prefix_len,
+                                        (const __nv_bfloat16*)k_rot, (const __nv_bfloat16*)v_rot,
+                                        (__nv_bfloat16*)ctx->attn_out,
+                                        (__nv_bfloat16*)ctx->attn_out + ctx->attn_lo_offset, st->softmax_scale, s));
+    else
+      CASCADE_TRY(launch_tree_attn_f32(ctx, tree, (const float*)ctx->q_rot, (const float*)L.k_prefix,
+                                       (const float*)L.v_prefix, st->prefix_cap, st->prefix_len, (const float*)k_rot,
+                                       (const float*)v_rot, (float*)ctx->attn_out, st->softmax_scale, s));
+    // output projection, residual, MLP norm
+    CASCADE_TRY(project(ctx, L.wo, sh.h, sh.Hq * sh.D, M, true, K_GEMM_O, &pr, s));
+    CASCADE_TRY(resid_norm<E>(ctx, T, nullptr, nullptr, &pr, L.gamma_mlp, st->eps, nullptr, K_RESID_NORM, s));
+    // gate and up stacked in memory: one projection
+    if ((const char*)L.w_up != (const char*)L.w_gate + (size_t)sh.ffn * sh.h * es) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+    CASCADE_TRY(project(ctx, L.w_gate, 2 * sh.ffn, sh.h, M, false, K_GEMM_GATE_UP, &pr, s));
+    {
+      const bool bf16 = sh.dtype == CASCADE_BF16;
+      KernelScope ks(ctx, K_SWIGLU, s);
+      k_swiglu<<<dim3(cascade_detail::ceil_div(sh.ffn, 4 * kRowThreads), M), kRowThreads, 0, s>>>(
+          ctx->gemm_out, pr.n_slices, pr.slice_stride, sh.ffn, bf16 ? ctx->act_hi : nullptr,
+          bf16 ? ctx->act_hi + ctx->act_lo_offset : nullptr, bf16 ? nullptr : ctx->act_f32);
+    }
+    CASCADE_CUDA_TRY(cudaGetLastError());
+    CASCADE_TRY(project(ctx, L.w_down, sh.h, sh.ffn, M, false, K_GEMM_DOWN, &pr, s));
+  }
+  // the last MLP output joins the residual stream; x is then the input of the final norm
+  return resid_norm<E>(ctx, T, nullptr, nullptr, &pr, nullptr, st->eps, st->hidden_out, K_RESID_ADD, s);
+}
+
+}  // namespace
+
+int run_layers(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, cudaStream_t s) {
+  if (ctx->shape.ffn <= 0 || ctx->x == nullptr) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (st->layers == nullptr || st->embed == nullptr || st->prefix_len == nullptr) return CASCADE_ERR_INVALID_ARG;
+  if (!(st->rope_base > 1.f) || !(st->softmax_scale > 0.f) || !(st->eps >= 0.f)) return CASCADE_ERR_INVALID_ARG;
+  if (st->prefix_cap < 0 || st->prefix_cap > ctx->shape.P_max) return CASCADE_ERR_INVALID_ARG;
+  if (ctx->shape.dtype == CASCADE_BF16) return run_layers_t<__nv_bfloat16>(ctx, tree, st, s);
+  return run_layers_t<float>(ctx, tree, st, s);
+}

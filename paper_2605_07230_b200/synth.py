@@ -339,3 +339,27 @@ def tail_inputs(w: Workload, rng, parent, noise: float = 0.15):
 def uniforms(rng, B: int, T: int) -> np.ndarray:
     """Pre-drawn acceptance draws r ~ U[0,1) (the verification rule's `random()` made an input)."""
     return rng.random((B, T), dtype=np.float32)
+
+
+def layer_step_inputs(w: Workload, rng, parent, n_layers: int = 1):
+    """Inputs of a verification step that runs through decoder layers: the clustered codebook as token
+    embedding and (tied) LM head, `n_layers` sets of N(0, 0.02) layer weights, an N(0,1) prefix KV cache
+    per layer (independent for the cond and uncond rows), stand-in drafter tokens and probabilities,
+    uniforms.  Everything is returned in the values the workload's element type can hold."""
+    T = len(parent)
+    R, H, D, P = 2 * w.B, w.n_heads, w.head_dim, w.prefix_len
+    E = quantize(clustered_codebook(rng, w.V, w.h, w.n_clusters, w.sigma), w.dtype)
+    layers = []
+    caches = []
+    for _ in range(n_layers):
+        lw = layer_weights(rng, w.h, H, D, w.ffn)
+        for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"):
+            setattr(lw, name, quantize(getattr(lw, name), w.dtype))
+        layers.append(lw)
+        caches.append((quantize(rng.standard_normal((R, P, H, D), dtype=np.float32), w.dtype),
+                       quantize(rng.standard_normal((R, P, H, D), dtype=np.float32), w.dtype)))
+    tok, p = cluster_drafter(rng, parent, w.B, w.V, w.n_clusters)
+    gamma = (1.0 + 0.1 * rng.standard_normal(w.h, dtype=np.float32)).astype(np.float32)
+    return dict(embed=E, w_head=E, layers=layers, k_prefix=[c[0] for c in caches], v_prefix=[c[1] for c in caches],
+                gamma_final=gamma, tok=tok, draft_p=p, uniforms=uniforms(rng, w.B, T),
+                prefix_len=np.full(R, P, np.int32))

@@ -129,3 +129,86 @@ class PiecesWorkload:
         w, T = self.w, self.T
         return {"lm_head": 2.0 * w.B * T * w.h * w.V,
                 "tree_attn": 4.0 * 2 * w.B * w.n_heads * T * (w.prefix_len + T) * w.head_dim}
+
+
+class LayerWorkload:
+    """The whole verification step through `n_layers` decoder layers: token embedding, layers (tree
+    attention over each layer's prefix cache), final norm, LM head with guidance, relaxed acceptance,
+    path selection.  `n_sets` copies of the weights and caches live at their own addresses (a benchmark
+    rotates through them so that a step never finds its operands in the L2)."""
+
+    def __init__(self, w: synth.Workload, n_layers: int = 1, device="cuda:0", n_sets: int = 1,
+                 keep_logits: bool = False, select_mode: int = cb.SELECT_LONGEST, flags: int = cb.USE_I | cb.USE_C):
+        self.w, self.device, self.n_layers = w, device, n_layers
+        self.parent = w.parent()
+        T = self.T = len(self.parent)
+        self.ctx = cb.Context(cb.BF16 if w.dtype == "bf16" else cb.F32, w.B, T, max(w.prefix_len, 1), w.h, w.n_heads,
+                              w.n_heads, w.head_dim, w.V, w.ffn)
+        self.tree = cb.Tree(self.ctx, self.parent)
+        self.params = cb.Params(w.tau_pos, w.tau_seq, w.tvd_budget, flags)
+        rng = np.random.default_rng(w.seed)
+        self.host = synth.layer_step_inputs(w, rng, self.parent, n_layers)
+        self.sets = [self._make_set(self.host if i == 0 else self._fresh_step(i), keep_logits, select_mode)
+                     for i in range(n_sets)]
+
+    def _fresh_step(self, i):
+        rng = np.random.default_rng(self.w.seed * 1000 + i)
+        tok, p = synth.cluster_drafter(rng, self.parent, self.w.B, self.w.V, self.w.n_clusters)
+        return dict(self.host, tok=tok, draft_p=p, uniforms=synth.uniforms(rng, self.w.B, self.T))
+
+    def _make_set(self, host, keep_logits, select_mode) -> DeviceStep:
+        w, T, dev, B = self.w, self.T, self.device, self.w.B
+        el = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        f32 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        d = dict(embed=to_device(host["embed"], w.dtype, dev), gamma_final=f32(host["gamma_final"]),
+                 prefix_len=f32(host["prefix_len"]), tok=f32(host["tok"]), draft_p=f32(host["draft_p"]),
+                 uniforms=f32(host["uniforms"]))
+        layers = []
+        for li, lw in enumerate(host["layers"]):
+            # q/k/v and gate/up stacked in memory: the library runs each group as one projection
+            qkv = to_device(np.concatenate([lw.wq, lw.wk, lw.wv], 0), w.dtype, dev)
+            gu = to_device(np.concatenate([lw.w_gate, lw.w_up], 0), w.dtype, dev)
+            hd = w.n_heads * w.head_dim
+            layers.append(dict(gamma_attn=f32(lw.gamma_attn), wq=qkv[:hd], wk=qkv[hd:2 * hd], wv=qkv[2 * hd:],
+                               wo=to_device(lw.wo, w.dtype, dev), gamma_mlp=f32(lw.gamma_mlp), w_gate=gu[:w.ffn],
+                               w_up=gu[w.ffn:], w_down=to_device(lw.w_down, w.dtype, dev),
+                               k_prefix=to_device(host["k_prefix"][li], w.dtype, dev),
+                               v_prefix=to_device(host["v_prefix"][li], w.dtype, dev), _keep=(qkv, gu)))
+        d["layers"] = layers
+        o = dict(
+            accept=torch.zeros((B, T), dtype=torch.uint8, device=dev),
+            path_nodes=torch.zeros((B, self.tree.depth + 1), dtype=torch.int32, device=dev),
+            path_len=torch.zeros(B, dtype=torch.int32, device=dev),
+            q_relaxed=torch.zeros((B, T), device=dev), tvd_out=torch.zeros((B, T), device=dev),
+            tvd_used=torch.zeros(B, device=dev), near_count=torch.zeros(B, dtype=torch.int32, device=dev),
+            feat=torch.zeros((B, T, w.h), device=dev), scores=torch.zeros((B, max(self.tree.num_pairs, 1)), device=dev),
+            row_lse=torch.zeros((B, T), device=dev), hidden_out=torch.zeros((2 * B, T, w.h), device=dev),
+            k_tree_out=torch.zeros((self.n_layers, 2 * B, T, w.n_heads, w.head_dim), dtype=el, device=dev),
+            v_tree_out=torch.zeros((self.n_layers, 2 * B, T, w.n_heads, w.head_dim), dtype=el, device=dev))
+        if keep_logits or w.dtype != "bf16":
+            o["logits"] = torch.zeros((B, T, w.V), device=dev)
+        step = cb.make_step(
+            layers=[{k: v for k, v in l.items() if k != "_keep"} for l in layers], embed=d["embed"],
+            gamma_final=d["gamma_final"], w_head=d["embed"], prefix_cap=w.prefix_len, prefix_len=d["prefix_len"],
+            eps=w.eps, rope_base=w.rope_base, softmax_scale=float(1.0 / np.sqrt(w.head_dim)), cfg_scale=w.cfg_scale,
+            temperature=1.0, tok=d["tok"], draft_p=d["draft_p"], uniforms=d["uniforms"], params=self.params,
+            select_mode=select_mode, accept=o["accept"], path_nodes=o["path_nodes"], path_len=o["path_len"],
+            q_relaxed=o["q_relaxed"], tvd_out=o["tvd_out"], tvd_used=o["tvd_used"], near_count=o["near_count"],
+            logits=o.get("logits"), feat=o["feat"], scores=o["scores"], row_lse=o["row_lse"],
+            hidden_out=o["hidden_out"], k_tree_out=o["k_tree_out"], v_tree_out=o["v_tree_out"])
+        return DeviceStep(host=host, dev=d, out=o, step=step)
+
+    def run(self, i: int = 0) -> DeviceStep:
+        s = self.sets[i % len(self.sets)]
+        cb.cascade_verify_step(self.ctx, self.tree, s.step)
+        return s
+
+    def close(self):
+        self.tree.close()
+        self.ctx.close()
+
+    def weight_bytes(self) -> dict:
+        w = self.w
+        e = 2 if w.dtype == "bf16" else 4
+        hd = w.n_heads * w.head_dim
+        return {"layer": (3 * hd * w.h + w.h * hd + 3 * w.ffn * w.h) * e * self.n_layers, "lm_head": w.V * w.h * e}
