@@ -1,9 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the CASCADE tree-verification step on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload janus|lumina|toy|mini] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload janus|lumina|toy|mini] [--mode layer|pieces]
+                    [--impl ours|reference]
 
-One "step" is one pass of the whole verification hot path over one synthetic batch.  Prints ONE JSON
+One "step" is one pass of the whole verification hot path over one synthetic batch: the tree tokens go
+through one decoder layer (embedding, q/k/v, rotary, tree attention over the prefix cache, output
+projection, SwiGLU MLP), the final norm, the LM head with guidance, relaxed acceptance and path selection
+(`--mode pieces` runs the four named pieces on stand-alone inputs without the layer's projections).  Prints ONE JSON
 line: verify-steps/s (device-timed with CUDA events, inputs resident in HBM), the same through the
 host-buffer C-ABI entry (`e2e`), the roofline of the dominant kernel measured live with CUDA events, the
 CPU checker timed on the host cores (`cpu_baseline`), and the SM clocks seen under load.
@@ -90,10 +94,16 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
-def oracle_step(w, parent, host):
+def oracle_step(w, parent, host, mode):
     """One whole verification step on the CPU checker (same inputs as the device step)."""
     from oracle import cascade_oracle as O
     scale = 1.0 / np.sqrt(w.head_dim)
+    if mode == "layer":
+        out = O.verify_step(host["embed"], host["layers"], host["gamma_final"], host["w_head"], host["tok"], parent,
+                            host["k_prefix"], host["v_prefix"], host["prefix_len"], host["draft_p"], host["uniforms"],
+                            w.n_heads, w.head_dim, w.eps, w.rope_base, w.cfg_scale, 1.0, w.tau_pos, w.tau_seq,
+                            w.tvd_budget, kv_bf16=w.dtype == "bf16")
+        return out["accept"]
     O.tree_attention(host["q"], host["k_prefix"], host["v_prefix"], host["prefix_len"], host["k_tree"],
                      host["v_tree"], parent, scale)
     head, res = O.verify_tail(host["hidden"], host["gamma_final"], w.eps, host["w_head"], w.cfg_scale, 1.0,
@@ -102,11 +112,11 @@ def oracle_step(w, parent, host):
     return res
 
 
-def time_oracle(w, parent, host, budget_s=25.0, max_steps=3):
+def time_oracle(w, parent, host, mode, budget_s=25.0, max_steps=3):
     t0 = time.perf_counter()
     n = 0
     while n < max_steps and (n == 0 or (time.perf_counter() - t0) * (n + 1) / n < budget_s):
-        oracle_step(w, parent, host)
+        oracle_step(w, parent, host, mode)
         n += 1
     dt = time.perf_counter() - t0
     try:
@@ -117,10 +127,12 @@ def time_oracle(w, parent, host, budget_s=25.0, max_steps=3):
     return n / dt, n, cores
 
 
-def host_inputs(w):
+def host_inputs(w, mode):
     from paper_2605_07230_b200 import synth
     parent = w.parent()
     rng = np.random.default_rng(w.seed)
+    if mode == "layer":
+        return parent, synth.layer_step_inputs(w, rng, parent, 1)
     host = {}
     host.update(synth.attention_inputs(w, rng, len(parent)))
     host.update(synth.tail_inputs(w, rng, parent))
@@ -132,13 +144,13 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    parent, host = host_inputs(w)
+    parent, host = host_inputs(w, args.mode)
     for _ in range(min(args.warmup, 1)):
-        oracle_step(w, parent, host)
+        oracle_step(w, parent, host, args.mode)
     steps = max(1, min(args.steps, 3))
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle_step(w, parent, host)
+        oracle_step(w, parent, host, args.mode)
     dt = time.perf_counter() - t0
     try:
         from threadpoolctl import threadpool_info
@@ -151,7 +163,7 @@ def run_reference(args, w):
         "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "tree_rows": len(parent), "prefix_len": w.prefix_len, "V": w.V,
-                   "h": w.h, "note": "CPU checker (numpy fp64), whole step; steps capped at 3"},
+                   "h": w.h, "mode": args.mode, "note": "CPU checker (numpy fp64), whole step; steps capped at 3"},
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{steps} whole step(s) of the {w.name} workload"},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -166,6 +178,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default="janus")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="layer", choices=["layer", "pieces"],
+                    help="layer: the step runs through one decoder layer; pieces: the four named pieces alone")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every step from Python instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets (0 = enough to exceed the L2 per step)")
@@ -180,7 +194,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2605_07230_b200 import binding as cb
-    from paper_2605_07230_b200.workload import PiecesWorkload
+    from paper_2605_07230_b200.workload import LayerWorkload, PiecesWorkload
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -194,9 +208,14 @@ def main():
     # enough rotating copies of the inputs that a step never finds its operands in the 126 MB L2
     parent = w.parent()
     T = len(parent)
-    per_set = (w.V * w.h + 2 * 2 * w.B * (w.prefix_len + T) * w.n_heads * w.head_dim) * 2
+    hd = w.n_heads * w.head_dim
+    layer_bytes = (4 * hd * w.h + 3 * w.ffn * w.h) * 2 if args.mode == "layer" else 0
+    per_set = (w.V * w.h + 2 * 2 * w.B * (w.prefix_len + T) * hd) * 2 + layer_bytes
     n_sets = args.sets or max(2, int(np.ceil(3 * 126e6 / per_set)))
-    wl = PiecesWorkload(w, device=dev, n_sets=n_sets)
+    if args.mode == "layer":
+        wl = LayerWorkload(w, n_layers=1, device=dev, n_sets=n_sets)
+    else:
+        wl = PiecesWorkload(w, device=dev, n_sets=n_sets)
     K, W = args.steps, max(args.warmup, 3)
 
     stream = torch.cuda.Stream()
@@ -290,26 +309,38 @@ def main():
 
     h2d = 3 * w.B * T * 4
     d2h = w.B * T + w.B * (wl.tree.depth + 1) * 4 + w.B * 4
-    alg_b, alg_f = wl.algorithmic_bytes(), wl.algorithmic_flops()
+    # algorithmic bytes per launch of each streaming kernel: its weight matrix (or K/V) once + operands
+    e = 2 if w.dtype == "bf16" else 4
+    R = 2 * w.B
+    act = R * T * e
+    alg_b = {
+        "tree_attn": R * (w.prefix_len + T) * hd * 2 * e + 2 * R * T * hd * e,
+        "gemm_head": w.V * w.h * e + R * T * w.h * e,
+        "gemm_qkv": 3 * hd * w.h * e + act * w.h,
+        "gemm_o": w.h * hd * e + act * hd,
+        "gemm_gate_up": 2 * w.ffn * w.h * e + act * w.h,
+        "gemm_down": w.h * w.ffn * e + act * w.ffn,
+    }
+    alg_f = {"gemm_head": 2.0 * w.B * T * w.h * w.V}
     per_kernel = {k: {"us": 1e3 * v[0] / v[1], "launches_per_step": v[1] / kt_steps} for k, v in timing.items()}
     step_us_kernels = sum(1e3 * v[0] for v in timing.values()) / kt_steps
-    dom = max(timing, key=lambda k: timing[k][0])
-    head_us = per_kernel.get("gemm_head", {}).get("us")
-    attn_us = per_kernel.get("tree_attn", {}).get("us")
-    roofline = None
-    if head_us:
-        ach = alg_b["lm_head"] / (head_us * 1e-6) / 1e9
-        roofline = {"kernel": "gemm_head (LM head, tcgen05)", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-                    "us_per_launch": head_us, "algorithmic_bytes": alg_b["lm_head"],
-                    "tensor_tflops": alg_f["lm_head"] / (head_us * 1e-6) / 1e12,
-                    "tensor_frac_of_bf16_peak": alg_f["lm_head"] / (head_us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
-    extra = {}
-    if attn_us:
-        ach = alg_b["tree_attn"] / (attn_us * 1e-6) / 1e9
-        extra["tree_attn"] = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                              "frac": ach / peaks["hbm_gbs"], "us_per_launch": attn_us,
-                              "algorithmic_bytes": alg_b["tree_attn"]}
+    dom = max((k for k in timing if k in alg_b), key=lambda k: timing[k][0])
+    def roof(k):
+        us = per_kernel[k]["us"]
+        ach = alg_b[k] / (us * 1e-6) / 1e9
+        d = {"kernel": k, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+             "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"], "us_per_launch": us,
+             "algorithmic_bytes": alg_b[k]}
+        if k in alg_f:
+            d["tensor_tflops"] = alg_f[k] / (us * 1e-6) / 1e12
+            d["tensor_frac_of_bf16_peak"] = d["tensor_tflops"] / peaks["bf16_tflops"]
+        return d
+    roofline = roof(dom)
+    extra = {k: roof(k) for k in per_kernel if k in alg_b and k != dom}
+    # the whole step against the bytes it has to stream once
+    step_bytes = sum(alg_b[k] for k in per_kernel if k in alg_b)
+    step_roof = {"algorithmic_bytes": step_bytes, "floor_us": step_bytes / peaks["hbm_gbs"] / 1e3,
+                 "frac_of_hbm_floor": step_bytes / peaks["hbm_gbs"] / 1e3 / (1e3 * ms / done)}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": done, "warmup": W,
@@ -317,7 +348,10 @@ def main():
         "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "tree_rows": T, "prefix_len": w.prefix_len, "V": w.V, "h": w.h,
                    "heads": w.n_heads, "head_dim": w.head_dim, "cfg_scale": w.cfg_scale,
-                   "step": "tree attention + final norm + LM head/CFG + relaxed acceptance + path selection",
+                   "mode": args.mode,
+                   "step": ("embedding + one decoder layer (q/k/v, rotary, tree attention, output projection, SwiGLU MLP) + "
+                            if args.mode == "layer" else "") +
+                           "tree attention + final norm + LM head/CFG + relaxed acceptance + path selection",
                    "l2": f"inputs rotate over {n_sets} sets of {per_set / 1e6:.0f} MB (> 126 MB L2 between reuses)",
                    "cuda_graph": graph is not None, "parallelism": "replicas" if world > 1 else "single"},
         "accepted_tokens_per_step": alpha_sum / (e2e_steps * w.B),
@@ -326,11 +360,11 @@ def main():
         "launches_per_step": launches_per_step,
         "kernels_us": {k: round(v["us"], 3) for k, v in sorted(per_kernel.items())},
         "kernel_time_per_step_us": step_us_kernels, "dominant_kernel": dom,
-        "roofline": roofline, "roofline_other": extra,
+        "roofline": roofline, "roofline_other": extra, "step_roofline": step_roof,
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        v, n, cores = time_oracle(w, parent, wl.sets[0].host)
+        v, n, cores = time_oracle(w, parent, wl.sets[0].host, args.mode, max_steps=1 if args.mode == "layer" else 3)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{n} whole step(s) of the {w.name} workload"}
     print(json.dumps(line))

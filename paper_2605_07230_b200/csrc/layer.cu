@@ -40,7 +40,41 @@ __device__ __forceinline__ void put_operand(__nv_bfloat16* hi, __nv_bfloat16* lo
   }
 }
 
-// One CTA per row m = r * T + j of the CFG pair.
+__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+  const uint2 r = *reinterpret_cast<const uint2*>(p);
+  return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u), __uint_as_float(r.y << 16),
+                     __uint_as_float(r.y & 0xffff0000u));
+}
+__device__ __forceinline__ void add4(float4& a, const float4 b) {
+  a.x += b.x;
+  a.y += b.y;
+  a.z += b.z;
+  a.w += b.w;
+}
+// four consecutive operand values
+__device__ __forceinline__ void put_operand4(__nv_bfloat16* hi, __nv_bfloat16* lo, float* f32, size_t i, const float4 a) {
+  if (hi != nullptr) {
+    const float v[4] = {a.x, a.y, a.z, a.w};
+    uint32_t h[2], l[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * k]), h1 = __float2bfloat16_rn(v[2 * k + 1]);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(v[2 * k] - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(v[2 * k + 1] - __bfloat162float(h1));
+      h[k] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      l[k] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    *reinterpret_cast<uint2*>(hi + i) = make_uint2(h[0], h[1]);
+    *reinterpret_cast<uint2*>(lo + i) = make_uint2(l[0], l[1]);
+  } else {
+    *reinterpret_cast<float4*>(f32 + i) = a;
+  }
+}
+
+constexpr int kRowChunks = 8;  // float4 chunks of a row a thread keeps in registers (rows up to 8192 elements)
+
+// One CTA per row m = r * T + j of the CFG pair.  h is a multiple of 4.
 //   x[m] (+)= ...: embed != null: x[m] = embed[tok[b, j]]            (first layer)
 //                  else          x[m] += sum_s slices[s][m]          (output of the previous projection)
 //   operand[m] = RMSNorm(x[m], gamma)                                (skipped when gamma == null)
@@ -57,83 +91,128 @@ __global__ void __launch_bounds__(kRowThreads) k_resid_norm(float* __restrict__ 
   const int m = blockIdx.x;
   const int r = m / T, j = m - r * T, b = r % B;
   float* xr = x + (size_t)m * h;
-  float ss = 0.f;
-  for (int i = threadIdx.x; i < h; i += kRowThreads) {
-    float v;
-    if (embed != nullptr) {
-      v = elem_to_float(embed, (size_t)tok[(size_t)b * T + j] * h + i);
+  const E* er = embed != nullptr ? embed + (size_t)tok[(size_t)b * T + j] * h : nullptr;
+  const int n4 = h / 4;
+  auto value = [&](int c) {  // element chunk c of the updated row
+    float4 v;
+    if (er != nullptr) {
+      v = load4(er + 4 * c);
     } else {
-      v = xr[i];
-      for (int s = 0; s < n_slices; ++s) v += slices[(size_t)s * slice_stride + (size_t)m * h + i];
+      v = load4(xr + 4 * c);
+      for (int s = 0; s < n_slices; ++s) add4(v, load4(slices + (size_t)s * slice_stride + (size_t)m * h + 4 * c));
     }
-    xr[i] = v;
-    if (x_copy != nullptr) x_copy[(size_t)m * h + i] = v;
-    ss += v * v;
+    return v;
+  };
+  float4 keep[kRowChunks];
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < kRowChunks; ++k) {
+    const int c = threadIdx.x + k * kRowThreads;
+    if (c < n4) {
+      keep[k] = value(c);
+      ss += keep[k].x * keep[k].x + keep[k].y * keep[k].y + keep[k].z * keep[k].z + keep[k].w * keep[k].w;
+      *reinterpret_cast<float4*>(xr + 4 * c) = keep[k];
+      if (x_copy != nullptr) *reinterpret_cast<float4*>(x_copy + (size_t)m * h + 4 * c) = keep[k];
+    }
+  }
+  for (int c = threadIdx.x + kRowChunks * kRowThreads; c < n4; c += kRowThreads) {  // longer rows: via memory
+    const float4 v = value(c);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    *reinterpret_cast<float4*>(xr + 4 * c) = v;
+    if (x_copy != nullptr) *reinterpret_cast<float4*>(x_copy + (size_t)m * h + 4 * c) = v;
   }
   if (gamma == nullptr) return;
   ss = block_sum(ss, red);
   const float rs = rsqrtf(ss / h + eps);
-  for (int i = threadIdx.x; i < h; i += kRowThreads) put_operand(a_hi, a_lo, a_f32, (size_t)m * h + i, xr[i] * rs * gamma[i]);
+  auto emit = [&](int c, const float4 v) {
+    const float4 g = load4(gamma + 4 * c);
+    put_operand4(a_hi, a_lo, a_f32, (size_t)m * h + 4 * c, make_float4(v.x * rs * g.x, v.y * rs * g.y, v.z * rs * g.z, v.w * rs * g.w));
+  };
+#pragma unroll
+  for (int k = 0; k < kRowChunks; ++k) {
+    const int c = threadIdx.x + k * kRowThreads;
+    if (c < n4) emit(c, keep[k]);
+  }
+  for (int c = threadIdx.x + kRowChunks * kRowThreads; c < n4; c += kRowThreads) emit(c, load4(xr + 4 * c));
 }
 
 // q, k, v = sum of the projection's slices; rotary embedding (half-split pairing: (x[i], x[i + D/2]) turned
 // by pos * base^(-2i/D)) on q and k at pos = prefix_len[r] + depth[j]; results in the attention's
-// element type.  grid (T, R), one thread per (head, pair index).
+// element type.  grid (T, R): one position per CTA, so its D/2 (cos, sin) pairs are computed once into
+// shared memory.  D is a multiple of 8.
 template <typename E>
 __global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restrict__ slices, int n_slices,
                                                             long long slice_stride, int T, int Hq, int Hkv, int D,
                                                             const int32_t* __restrict__ prefix_len,
                                                             const int32_t* __restrict__ depth, float rope_base,
                                                             E* __restrict__ q, E* __restrict__ k, E* __restrict__ v) {
+  __shared__ float s_cos[128], s_sin[128];  // D <= 256
   const int j = blockIdx.x, r = blockIdx.y;
   const size_t m = (size_t)r * T + j;
   const int n_cols = (Hq + 2 * Hkv) * D, half = D / 2;
   const float pos = (float)(prefix_len[r] + depth[j]);
-  auto col = [&](int c) {
-    float a = 0.f;
-    for (int s = 0; s < n_slices; ++s) a += slices[(size_t)s * slice_stride + m * n_cols + c];
+  for (int i = threadIdx.x; i < half; i += kRowThreads) {
+    const float inv_freq = powf(rope_base, -2.f * (float)i / (float)D);
+    sincosf(pos * inv_freq, &s_sin[i], &s_cos[i]);
+  }
+  __syncthreads();
+  auto col4 = [&](int c) {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < n_slices; ++s) add4(a, load4(slices + (size_t)s * slice_stride + m * n_cols + c));
     return a;
   };
-  auto store = [](E* dst, size_t i, float val) {
-    if constexpr (sizeof(E) == 2) dst[i] = __float2bfloat16_rn(val);
-    else dst[i] = val;
+  auto store4 = [](E* dst, size_t i, const float4 a) {
+    if constexpr (sizeof(E) == 2) {
+      const __nv_bfloat16 b0 = __float2bfloat16_rn(a.x), b1 = __float2bfloat16_rn(a.y), b2 = __float2bfloat16_rn(a.z),
+                          b3 = __float2bfloat16_rn(a.w);
+      *reinterpret_cast<uint2*>(dst + i) =
+          make_uint2((uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16),
+                     (uint32_t)__bfloat16_as_ushort(b2) | ((uint32_t)__bfloat16_as_ushort(b3) << 16));
+    } else {
+      *reinterpret_cast<float4*>(dst + i) = a;
+    }
   };
-  // rotated pairs of q and k
-  for (int t = threadIdx.x; t < (Hq + Hkv) * half; t += kRowThreads) {
-    const int head = t / half, i = t - head * half;
+  // rotated pairs of q and k, four pair indices per thread and step
+  const int q4 = half / 4;
+  for (int t = threadIdx.x; t < (Hq + Hkv) * q4; t += kRowThreads) {
+    const int head = t / q4, i = (t - head * q4) * 4;
     const int c0 = head * D + i;  // q heads first, then k heads: same column order as the projection
-    const float x1 = col(c0), x2 = col(c0 + half);
-    const float inv_freq = powf(rope_base, -2.f * (float)i / (float)D);
-    float sn, cs;
-    sincosf(pos * inv_freq, &sn, &cs);
-    const float y1 = x1 * cs - x2 * sn, y2 = x2 * cs + x1 * sn;
+    const float4 x1 = col4(c0), x2 = col4(c0 + half);
+    const float4 cs = load4(s_cos + i), sn = load4(s_sin + i);
+    const float4 y1 = make_float4(x1.x * cs.x - x2.x * sn.x, x1.y * cs.y - x2.y * sn.y, x1.z * cs.z - x2.z * sn.z,
+                                  x1.w * cs.w - x2.w * sn.w);
+    const float4 y2 = make_float4(x2.x * cs.x + x1.x * sn.x, x2.y * cs.y + x1.y * sn.y, x2.z * cs.z + x1.z * sn.z,
+                                  x2.w * cs.w + x1.w * sn.w);
     if (head < Hq) {
       const size_t o = (m * Hq + head) * D + i;
-      store(q, o, y1);
-      store(q, o + half, y2);
+      store4(q, o, y1);
+      store4(q, o + half, y2);
     } else {
       const size_t o = (m * Hkv + (head - Hq)) * D + i;
-      store(k, o, y1);
-      store(k, o + half, y2);
+      store4(k, o, y1);
+      store4(k, o + half, y2);
     }
   }
-  for (int t = threadIdx.x; t < Hkv * D; t += kRowThreads) store(v, m * Hkv * D + t, col((Hq + Hkv) * D + t));
+  for (int t = threadIdx.x; t < Hkv * D / 4; t += kRowThreads) store4(v, m * Hkv * D + 4 * t, col4((Hq + Hkv) * D + 4 * t));
 }
 
 // act = silu(gate) * up from the slices of the fused gate/up projection ([.., 2*ffn]: gate then up).
+// ffn is a multiple of 4.
 __global__ void __launch_bounds__(kRowThreads) k_swiglu(const float* __restrict__ slices, int n_slices,
                                                         long long slice_stride, int ffn,
                                                         __nv_bfloat16* __restrict__ a_hi,
                                                         __nv_bfloat16* __restrict__ a_lo, float* __restrict__ a_f32) {
   const size_t m = blockIdx.y;
-  for (int i = blockIdx.x * kRowThreads + threadIdx.x; i < ffn; i += gridDim.x * kRowThreads) {
-    float g = 0.f, u = 0.f;
+  for (int c = blockIdx.x * kRowThreads + threadIdx.x; c < ffn / 4; c += gridDim.x * kRowThreads) {
+    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
     for (int s = 0; s < n_slices; ++s) {
       const float* row = slices + (size_t)s * slice_stride + m * 2 * ffn;
-      g += row[i];
-      u += row[ffn + i];
+      add4(g, load4(row + 4 * c));
+      add4(u, load4(row + ffn + 4 * c));
     }
-    put_operand(a_hi, a_lo, a_f32, m * ffn + i, g / (1.f + expf(-g)) * u);
+    put_operand4(a_hi, a_lo, a_f32, m * ffn + 4 * c,
+                 make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
+                             g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w));
   }
 }
 
@@ -214,6 +293,9 @@ int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step*
         L.gamma_mlp == nullptr || L.w_gate == nullptr || L.w_up == nullptr || L.w_down == nullptr)
       return CASCADE_ERR_INVALID_ARG;
     if (st->prefix_cap > 0 && (L.k_prefix == nullptr || L.v_prefix == nullptr)) return CASCADE_ERR_INVALID_ARG;
+    if (((uintptr_t)L.gamma_attn | (uintptr_t)L.gamma_mlp | (uintptr_t)L.wq | (uintptr_t)L.wo | (uintptr_t)L.w_gate |
+         (uintptr_t)L.w_down | (uintptr_t)L.k_prefix | (uintptr_t)L.v_prefix) & 15u)
+      return CASCADE_ERR_INVALID_ARG;  // vector loads and TMA need 16-byte aligned bases
     // input norm (first layer: from the token embeddings; later: after adding the previous MLP output)
     CASCADE_TRY(resid_norm<E>(ctx, T, li == 0 ? st->embed : nullptr, st->tok, li == 0 ? nullptr : &pr, L.gamma_attn,
                               st->eps, nullptr, li == 0 ? K_EMBED_NORM : K_RESID_NORM, s));
@@ -251,7 +333,7 @@ int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step*
     {
       const bool bf16 = sh.dtype == CASCADE_BF16;
       KernelScope ks(ctx, K_SWIGLU, s);
-      k_swiglu<<<dim3(cascade_detail::ceil_div(sh.ffn, 4 * kRowThreads), M), kRowThreads, 0, s>>>(
+      k_swiglu<<<dim3(cascade_detail::ceil_div(sh.ffn / 4, kRowThreads), M), kRowThreads, 0, s>>>(
           ctx->gemm_out, pr.n_slices, pr.slice_stride, sh.ffn, bf16 ? ctx->act_hi : nullptr,
           bf16 ? ctx->act_hi + ctx->act_lo_offset : nullptr, bf16 ? nullptr : ctx->act_f32);
     }
