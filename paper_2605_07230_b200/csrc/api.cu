@@ -6,6 +6,7 @@
 
 #include "cascade_internal.h"
 #include "gemm_tc.h"
+#include "operand.cuh"
 #include "tmap.h"
 
 namespace cascade_detail {
@@ -52,8 +53,7 @@ int64_t carve(cascade_ctx* c, char* base) {
   cv.take(c->attn_unit_done, (int64_t)R * s.Hq * (t_pad / 64));
   c->head_m_pad = (int)align_up(BT, 128);
   if (s.dtype == CASCADE_BF16) {
-    c->head_lo_offset = (int64_t)c->head_m_pad * s.h;
-    cv.take(c->head_a_hi, 2 * c->head_lo_offset);
+    cv.take(c->head_a, operand_elems((int)BT, s.h));
     c->head_max_tiles = ceil_div(s.V, 128);
     cv.take(c->head_part, (int64_t)c->head_max_tiles * c->head_m_pad);
     cv.take(c->gemm_scratch, gemm_tc_scratch_floats(c->sm_count));
@@ -76,8 +76,7 @@ int64_t carve(cascade_ctx* c, char* base) {
     const int es = elem_size(s);
     cv.take(c->x, RT * s.h);
     if (s.dtype == CASCADE_BF16) {
-      c->act_lo_offset = align_up(RT * k_max, 128);
-      cv.take(c->act_hi, 2 * c->act_lo_offset);
+      cv.take(c->act, operand_elems((int)RT, (int)align_up(k_max, 64)));
     } else {
       cv.take(c->act_f32, RT * k_max);
     }
@@ -97,8 +96,7 @@ int64_t carve(cascade_ctx* c, char* base) {
     c->k_rot = p;
     cv.take(p, RT * s.Hkv * s.D * es);
     c->v_rot = p;
-    c->attn_lo_offset = s.dtype == CASCADE_BF16 ? align_up(RT * s.Hq * s.D, 128) : 0;
-    cv.take(p, (RT * s.Hq * s.D + c->attn_lo_offset) * es);
+    cv.take(p, s.dtype == CASCADE_BF16 ? operand_elems((int)RT, s.Hq * s.D) * 2 : RT * s.Hq * s.D * es);
     c->attn_out = p;
   }
   cv.take(c->st_tok, BT);
@@ -120,6 +118,7 @@ int validate_shape(const cascade_shape* s) {
   if (s->D != 64 && s->D != 128) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (s->Hq % s->Hkv != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (s->h % 64 != 0 || s->V % 8 != 0 || s->ffn % 8 != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (s->dtype == CASCADE_BF16 && s->ffn % 64 != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;  // GEMM K blocks of 64
   if ((int64_t)s->B * s->T_max > (1 << 20)) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   return CASCADE_OK;
 }
@@ -373,7 +372,7 @@ static int tree_attn_impl(cascade_ctx* ctx, const cascade_tree* tree, const void
     return launch_tree_attn_bf16(ctx, tree, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_prefix,
                                  (const __nv_bfloat16*)v_prefix, prefix_cap, prefix_len,
                                  (const __nv_bfloat16*)k_tree, (const __nv_bfloat16*)v_tree, (__nv_bfloat16*)out,
-                                 nullptr, softmax_scale, s);
+                                 false, softmax_scale, s);
   return launch_tree_attn_f32(ctx, tree, (const float*)q, (const float*)k_prefix, (const float*)v_prefix,
                               prefix_cap, prefix_len, (const float*)k_tree, (const float*)v_tree, (float*)out,
                               softmax_scale, s);

@@ -22,21 +22,29 @@
 // waiting) and writes the bf16 rows.  With one split the CTA writes the final rows itself.
 // Every mbarrier wait is bounded (error word + normal teardown on expiry).
 #include "cascade_internal.h"
+#include "operand.cuh"
 #include "ptx.cuh"
 #include "tmap.h"
 
 namespace {
 
-// 8 consecutive outputs as bf16 (and, if asked for, what the rounding dropped as a second bf16 vector)
-__device__ __forceinline__ void store8(__nv_bfloat16* out, __nv_bfloat16* out_lo, size_t at, const float* v) {
+// 8 consecutive outputs of (row m of R*T, column col of Hq*D): bf16 row-major, or -- for the output
+// projection that follows inside a decoder layer -- the bf16 pair (value, what the rounding dropped) in the
+// GEMM's staged operand layout
+template <typename Args>
+__device__ __forceinline__ void store8(const Args& p, int m, int col, int row_len, const float* v) {
   uint32_t hi[4], lo[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     hi[k] = ptx::pack_bf16x2(v[2 * k], v[2 * k + 1]);
     lo[k] = ptx::pack_bf16x2(v[2 * k] - __uint_as_float(hi[k] << 16), v[2 * k + 1] - __uint_as_float(hi[k] & 0xffff0000u));
   }
-  *reinterpret_cast<uint4*>(out + at) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-  if (out_lo != nullptr) *reinterpret_cast<uint4*>(out_lo + at) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  if (p.out_as_operand) {
+    *reinterpret_cast<uint4*>(p.out + operand_index(p.out_lay, m, col, 0)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(p.out + operand_index(p.out_lay, m, col, 1)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  } else {
+    *reinterpret_cast<uint4*>(p.out + (size_t)m * row_len + col) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+  }
 }
 
 constexpr int kD = 128;
@@ -57,7 +65,8 @@ struct AttnArgs {
   const int32_t* prefix_len;
   const uint64_t* anc;
   __nv_bfloat16* out;
-  __nv_bfloat16* out_lo;  // optional: bf16 remainder out - bf16(out), same layout (a later GEMM adds both parts)
+  int out_as_operand;     // 1: `out` receives the (R*T x Hq*D) matrix as a GEMM operand (bf16 pair, staged layout)
+  OperandLayout out_lay;
   float* part_o;
   float2* part_ml;
   float c;  // softmax_scale * log2(e)
@@ -365,13 +374,12 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       const float l = l_run * w0 + l1 * w1;
       if (p.splits == 1) {
         const float inv = 1.f / l;
-        const size_t at = (((size_t)r * p.T + j) * p.Hq + head) * kD;
 #pragma unroll
         for (int c = 0; c < kD / 8; ++c) {
           float v8[8];
 #pragma unroll
           for (int k = 0; k < 8; ++k) v8[k] = (o_acc[c * 8 + k] * w0 + x[c * 8 + k] * w1) * inv;
-          store8(p.out, p.out_lo, at + c * 8, v8);
+          store8(p, r * p.T + j, head * kD + c * 8, p.Hq * kD, v8);
         }
       } else {
         const size_t unit = ((size_t)r * p.Hq + head) * p.splits + split;
@@ -447,13 +455,12 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
   }
   const float inv = 1.f / l;
-  const size_t at = (((size_t)r * p.T + j) * p.Hq + head) * kD + d0;
 #pragma unroll
   for (int c = 0; c < kD / 16; ++c) {
     float v8[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) v8[k] = acc[8 * c + k] * inv;
-    store8(p.out, p.out_lo, at + c * 8, v8);
+    store8(p, r * p.T + j, head * kD + d0 + c * 8, p.Hq * kD, v8);
   }
 }
 
@@ -462,7 +469,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* q,
                           const __nv_bfloat16* kp, const __nv_bfloat16* vp, int prefix_cap,
                           const int32_t* prefix_len, const __nv_bfloat16* kt, const __nv_bfloat16* vt,
-                          __nv_bfloat16* out, __nv_bfloat16* out_lo, float scale, cudaStream_t s) {
+                          __nv_bfloat16* out, bool out_as_operand, float scale, cudaStream_t s) {
   const cascade_shape& sh = ctx->shape;
   if (sh.D != kD) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   const int T = tree->T, R = 2 * sh.B;
@@ -476,7 +483,8 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   a.prefix_len = prefix_len;
   a.anc = tree->d_anc;
   a.out = out;
-  a.out_lo = out_lo;
+  a.out_as_operand = out_as_operand ? 1 : 0;
+  a.out_lay = operand_layout(R * T, sh.Hq * kD);
   a.part_o = ctx->attn_part_o;
   a.part_ml = ctx->attn_part_ml;
   a.c = scale * 1.4426950408889634f;

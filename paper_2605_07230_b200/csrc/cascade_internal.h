@@ -73,8 +73,7 @@ struct cascade_ctx {
 
   // LM head
   int head_m_pad = 0;             // B*T_max rounded up to 128
-  __nv_bfloat16* head_a_hi = nullptr;  // [head_m_pad][h], followed by the remainder part [head_m_pad][h]
-  int64_t head_lo_offset = 0;          // elements from head_a_hi to the remainder part
+  __nv_bfloat16* head_a = nullptr;     // the head's activation operand (B*T x h) in the GEMM's staged layout
   int head_max_tiles = 0;
   float2* head_part = nullptr;    // [head_max_tiles][head_m_pad] (tile max, tile sum of exp)
   float* head_a_f32 = nullptr;    // [B*T_max][h] mixed operand (fp32 path)
@@ -93,8 +92,7 @@ struct cascade_ctx {
 
   // decoder layer activations (allocated when ffn > 0)
   float* x = nullptr;            // [R*T][h] residual stream, fp32
-  __nv_bfloat16* act_hi = nullptr;  // [R*T][max(h,ffn)] GEMM operand, high part; the remainder part follows at
-  int64_t act_lo_offset = 0;        // act_hi + act_lo_offset (elements)
+  __nv_bfloat16* act = nullptr;  // GEMM operand (R*T x max(h,ffn)) in the GEMM's staged layout (bf16 pair)
   float* act_f32 = nullptr;      // [R*T][max(h,ffn)] GEMM operand (fp32 path)
   float* gemm_out = nullptr;     // [slices][R*T][N] fp32 projection results, one matrix per K slice
   int64_t gemm_out_floats = 0;
@@ -102,8 +100,8 @@ struct cascade_ctx {
   void* q_rot = nullptr;         // [R,T,Hq,D] elem
   void* k_rot = nullptr;         // [R,T,Hkv,D] elem
   void* v_rot = nullptr;
-  void* attn_out = nullptr;      // [R,T,Hq,D] elem; bf16: followed by the rounding remainder, same shape
-  int64_t attn_lo_offset = 0;    // elements from attn_out to that remainder
+  void* attn_out = nullptr;      // fp32 path: [R,T,Hq,D] float; bf16 path: the output projection's operand
+                                 // (R*T x Hq*D, bf16 pair) in the GEMM's staged layout
 
   // staging for the host-buffer entry point
   int32_t* st_tok = nullptr;
@@ -203,7 +201,7 @@ int launch_tree_attn_f32(cascade_ctx* ctx, const cascade_tree* tree, const float
 int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* q,
                           const __nv_bfloat16* kp, const __nv_bfloat16* vp, int prefix_cap,
                           const int32_t* prefix_len, const __nv_bfloat16* kt, const __nv_bfloat16* vt,
-                          __nv_bfloat16* out, __nv_bfloat16* out_lo, float scale, cudaStream_t s);
+                          __nv_bfloat16* out, bool out_as_operand, float scale, cudaStream_t s);
 
 // head.cu (norm + mix producers, fp32 head) / gemm_tc.cu (tcgen05 GEMM)
 // cand_parent / cand_gparent (may be null) are cleared here; the head fills the entries that exist.

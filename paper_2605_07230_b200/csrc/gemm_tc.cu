@@ -22,7 +22,8 @@
 //         matrix and the consumer adds the S matrices.  Nothing waits inside the kernel; this is for
 //         weight matrices with so few tiles that each would be cut many times;
 //   * a TMA producer thread keeps a ring of [W rows x 64 | Ahi NB x 64 | Alo NB x 64] bf16 stages
-//     (128-byte swizzle) in flight, one thread issues the UMMAs (the high part and the remainder of the
+//     (128-byte swizzle) in flight -- the weights by tiled TMA loads, the activations, which their
+//     producers already store in the staged layout (operand.cuh), by one contiguous bulk copy --, one thread issues the UMMAs (the high part and the remainder of the
 //     activation operand accumulate into the same fp32 TMEM accumulator), and four epilogue warps
 //     drain one of two TMEM accumulator sets while the next tile is being accumulated into the other.
 //     The producer and issue loops are kept to a few dozen instructions per stage: a single thread
@@ -35,6 +36,7 @@
 // the normal teardown (TMEM is freed).
 #include "cascade_internal.h"
 #include "gemm_tc.h"
+#include "operand.cuh"
 #include "ptx.cuh"
 #include "tmap.h"
 
@@ -51,7 +53,8 @@ constexpr int kTileWBytes = kTileN * kSpan * 2;
 
 struct GemmArgs {
   int M, N, NB, n_mchunks, n_kb, stages, tmem_cols;
-  int has_lo;              // 0: the activation operand is exact in bf16 (no remainder part)
+  const __nv_bfloat16* A;  // activation operand in the staged layout of operand.cuh
+  long long a_chunk_elems; // elements of one row chunk of A (all its K blocks)
   int stash;               // 1: TMEM has room for a third accumulator set (partials of split tiles)
   long long units;         // n_tiles * n_kb
   int n_tiles;
@@ -122,7 +125,7 @@ struct SegmentWalk {
 // kHalves: accumulators (128 weight rows each) per work tile.  kSpans: 64-wide K spans per stage.
 template <int kHalves, int kSpans>
 __global__ void __launch_bounds__(kThreads, 1)
-k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_a, const GemmArgs p) {
+k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
   constexpr int kWSpanBytes = kHalves * kTileWBytes;  // weights of one span
   constexpr int kWBytes = kSpans * kWSpanBytes;       // weights of one stage: span after span
   extern __shared__ uint8_t smem_raw[];
@@ -136,7 +139,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const int a_span_bytes = (1 + p.has_lo) * p.NB * kSpan * 2;  // one span of the activations: hi block [, lo block]
+  const int a_span_bytes = 2 * p.NB * kSpan * 2;  // one span of the activations: hi block, lo block
   const int stage_bytes = kWBytes + kSpans * a_span_bytes;
 
   if (threadIdx.x == 0) {
@@ -151,7 +154,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     s_abort = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tm_w);
-    ptx::prefetch_tmap(&tm_a);
   }
   if (warp == 1) {
     ptx::tmem_alloc(&s_tmem_base, (uint32_t)p.tmem_cols);
@@ -173,7 +175,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
       Segment sg;
       bool ok = true;
       while (ok && walk.next(sg)) {
-        const int n0 = (sg.tile / n_mchunks) * (kHalves * kTileN), m0 = (sg.tile % n_mchunks) * NB;
+        const int n0 = (sg.tile / n_mchunks) * (kHalves * kTileN);
+        const __nv_bfloat16* a_chunk = p.A + (size_t)(sg.tile % n_mchunks) * p.a_chunk_elems;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
           if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.err)) {
             ok = false;
@@ -182,10 +185,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           uint8_t* stage = smem + s * stage_bytes;
           ptx::mbar_arrive_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
 #pragma unroll
-          for (int q = 0; q < kSpans; ++q) {
+          for (int q = 0; q < kSpans; ++q)
             ptx::tma_load_2d(stage + q * kWSpanBytes, &tm_w, (kb * kSpans + q) * kSpan, n0, &full_bar[s]);
-            ptx::tma_load_3d(stage + kWBytes + q * a_span_bytes, &tm_a, (kb * kSpans + q) * kSpan, m0, 0, &full_bar[s]);
-          }
+          // the activations of these K blocks are contiguous in the staged layout: one bulk copy
+          ptx::bulk_load(stage + kWBytes, a_chunk + (size_t)kb * (kSpans * 2 * NB * kSpan), (uint32_t)(kSpans * a_span_bytes),
+                         &full_bar[s]);
           if (++s == stages) {
             s = 0;
             ph ^= 1u;
@@ -229,7 +233,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
               for (int ks = 0; ks < kSpan / 16; ++ks) {
                 // advancing 16 K elements = 32 bytes = 2 descriptor units inside the swizzle span
                 ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + 2 * ks, idesc, (q | ks) == 0 ? accumulate : 1u);
-                if (p.has_lo) ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
+                ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
               }
             }
           }
@@ -491,9 +495,9 @@ int gemm_tc_pick_splits(int sm_count, int M, int N, int K, int max_splits) {
   return best;
 }
 
-int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* a_hi,
-                   int64_t lo_offset, int M, const GemmEpilogue& epi, int kernel_id, cudaStream_t s) {
-  if (K % 8 != 0 || M < 1 || N < 1 || lo_offset % 8 != 0) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* A, int M,
+                   const GemmEpilogue& epi, int kernel_id, cudaStream_t s) {
+  if (K % kSpan != 0 || M < 1 || N < 1) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (epi.part != nullptr && epi.part_ld < cascade_detail::ceil_div(N, kTileN)) return CASCADE_ERR_INVALID_ARG;
   if (epi.splits < 0 || (epi.splits > 1 && (epi.part != nullptr || epi.accumulate || epi.C == nullptr)))
     return CASCADE_ERR_INVALID_ARG;
@@ -503,8 +507,11 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   GemmArgs a;
   a.M = M;
   a.N = N;
-  a.n_mchunks = cascade_detail::ceil_div(M, 128);
-  a.NB = (int)cascade_detail::align_up(cascade_detail::ceil_div(M, a.n_mchunks), 16);
+  const OperandLayout lay = operand_layout(M, K);
+  a.n_mchunks = lay.n_chunks;
+  a.NB = lay.NB;
+  a.A = A;
+  a.a_chunk_elems = (long long)lay.n_kb * 2 * lay.NB * kSpan;
   a.epi = epi;
   a.sk_scratch = ctx->gemm_scratch;
   a.sk_flags = ctx->gemm_flags;
@@ -516,9 +523,8 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   // no faster on the stream and split the LM head of a 16384-token vocabulary over too few tiles.)
   const int halves = 1;
   const int budget = 227 * 1024 - 20 * 1024 - 1024;  // static shared + alignment slack
-  a.has_lo = lo_offset != 0;
-  const int span_bytes = halves * kTileWBytes + (1 + a.has_lo) * a.NB * kSpan * 2;
-  const int spans = budget / (2 * span_bytes) >= 3 ? 2 : 1;
+  const int span_bytes = halves * kTileWBytes + 2 * a.NB * kSpan * 2;
+  const int spans = (K % (2 * kSpan) == 0 && budget / (2 * span_bytes) >= 3) ? 2 : 1;
   const int stage_bytes = spans * span_bytes;
   a.stages = budget / stage_bytes;
   if (a.stages > kMaxStages) a.stages = kMaxStages;
@@ -535,11 +541,7 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   while (a.tmem_cols < (a.stash ? 3 : 2) * halves * a.NB) a.tmem_cols *= 2;
   const CUtensorMap* tw =
       get_tmap_2d_bf16(ctx, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(halves * kTileN), kSpan);
-  const uint64_t ad[3] = {(uint64_t)K, (uint64_t)M, a.has_lo ? 2u : 1u};
-  const uint64_t as[2] = {(uint64_t)K, a.has_lo ? (uint64_t)lo_offset : (uint64_t)K * M};
-  const uint32_t ab[3] = {kSpan, (uint32_t)a.NB, a.has_lo ? 2u : 1u};
-  const CUtensorMap* ta = get_tmap_bf16(ctx, a_hi, 3, ad, as, ab);
-  if (tw == nullptr || ta == nullptr) return CASCADE_ERR_CUDA;
+  if (tw == nullptr) return CASCADE_ERR_CUDA;
   const int smem = a.stages * stage_bytes + 1024;
   auto kern = spans == 2 ? k_gemm_tc<1, 2> : k_gemm_tc<1, 1>;
   static int configured_smem[2] = {0, 0};
@@ -561,7 +563,7 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   cfg.numAttrs = epi.splits == 0 ? 1 : 0;
   {
     KernelScope ks(ctx, kernel_id, s);
-    CASCADE_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, *tw, *ta, a));
+    CASCADE_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, *tw, a));
   }
   return CASCADE_OK;
 }

@@ -24,11 +24,11 @@ struct GemmEpilogue {
 };
 
 // C[m][n] = sum_k (a_hi[m][k] + a_lo[m][k]) * W[n][k] on the tensor cores (see gemm_tc.cu).
-// W [N][K] bf16; a_hi [M][K] bf16 and the remainder a_lo = a_hi + lo_offset elements (same layout;
-// lo_offset = 0: no remainder part, the operand is exact in bf16);
-// K a multiple of 8.  Uses the context's split-tile scratch: calls on one context must not overlap.
-int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* a_hi,
-                   int64_t lo_offset, int M, const GemmEpilogue& epi, int kernel_id, cudaStream_t s);
+// W [N][K] bf16 row-major; A: the M x K activation operand (bf16 high part + bf16 remainder) in the staged
+// layout of operand.cuh; K a multiple of 64.  Uses the context's split-tile scratch: calls on one context
+// must not overlap.
+int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const __nv_bfloat16* A, int M,
+                   const GemmEpilogue& epi, int kernel_id, cudaStream_t s);
 // Floats of scratch the split-tile hand-off needs for a device with `sm_count` SMs.
 int64_t gemm_tc_scratch_floats(int sm_count);
 // Number of K slices (splits >= 1) that keeps the SMs evenly busy for an [N][K] weight matrix.

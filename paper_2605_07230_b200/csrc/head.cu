@@ -2,10 +2,12 @@
 //
 // The head is linear, so W n_u + s (W n_c - W n_u) = W (n_u + s (n_c - n_u)): the mix is done here on
 // the [B*T, h] operand and the product runs once.  For the bf16 path the mixed operand is stored as a
-// bf16 high part plus a bf16 remainder (a = hi + lo to ~16 mantissa bits); the tensor-core GEMM adds
-// both products into one fp32 accumulator.
+// bf16 high part plus a bf16 remainder (a = hi + lo to ~16 mantissa bits), in the staged layout the
+// tensor-core GEMM copies straight into shared memory; the GEMM adds both products into one fp32
+// accumulator.
 #include "cascade_internal.h"
 #include "gemm_tc.h"
+#include "operand.cuh"
 
 namespace {
 
@@ -44,9 +46,8 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
                                                                  const float* __restrict__ gamma, float eps, float s,
                                                                  float inv_temp, float* __restrict__ feat,
                                                                  float* __restrict__ feat_norm,
-                                                                 __nv_bfloat16* __restrict__ a_hi,
-                                                                 __nv_bfloat16* __restrict__ a_lo,
-                                                                 float* __restrict__ a_f32,
+                                                                 __nv_bfloat16* __restrict__ a_op,
+                                                                 const OperandLayout lay, float* __restrict__ a_f32,
                                                                  float* __restrict__ cand_parent,
                                                                  float* __restrict__ cand_gparent) {
   __shared__ float red[kNormThreads / 32];
@@ -99,7 +100,7 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
       *reinterpret_cast<float4*>(feat + o) = make_float4(nc[0], nc[1], nc[2], nc[3]);
       *reinterpret_cast<float4*>(feat + o + 4) = make_float4(nc[4], nc[5], nc[6], nc[7]);
     }
-    if (a_hi != nullptr) {
+    if (a_op != nullptr) {
       uint32_t hi[4], lo[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -109,8 +110,9 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
         hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
         lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
       }
-      *reinterpret_cast<uint4*>(a_hi + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-      *reinterpret_cast<uint4*>(a_lo + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      // GEMM operand in its staged layout: 8 consecutive K elements stay one 16-byte piece
+      *reinterpret_cast<uint4*>(a_op + operand_index(lay, (int)m, 8 * i, 0)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(a_op + operand_index(lay, (int)m, 8 * i, 1)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     } else {
       *reinterpret_cast<float4*>(a_f32 + o) = make_float4(a[0], a[1], a[2], a[3]);
       *reinterpret_cast<float4*>(a_f32 + o + 4) = make_float4(a[4], a[5], a[6], a[7]);
@@ -169,8 +171,7 @@ int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bflo
     e.cand_parent = cand_parent;
     e.cand_gparent = cand_gparent;
   }
-  return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a_hi, ctx->head_lo_offset, sh.B * tree->T, e, K_GEMM_HEAD,
-                        s);
+  return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a, sh.B * tree->T, e, K_GEMM_HEAD, s);
 }
 
 int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidden_f32, const float* gamma, float eps,
@@ -180,16 +181,16 @@ int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidd
   dim3 grid(T, sh.B);
   KernelScope ks(ctx, K_FINAL_NORM_MIX, s);
   const bool bf16 = sh.dtype == CASCADE_BF16;
-  __nv_bfloat16* a_hi = bf16 ? ctx->head_a_hi : nullptr;
-  __nv_bfloat16* a_lo = bf16 ? ctx->head_a_hi + ctx->head_lo_offset : nullptr;
+  __nv_bfloat16* a_op = bf16 ? ctx->head_a : nullptr;
+  const OperandLayout lay = operand_layout(sh.B * T, sh.h);
   float* a_f32 = bf16 ? nullptr : ctx->head_a_f32;
   if (bf16 && !hidden_f32)
     k_final_norm_mix<__nv_bfloat16><<<grid, kNormThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(hidden), sh.B, T,
                                                                   sh.h, gamma, eps, cfg_scale, inv_temperature, feat,
-                                                                  feat_norm, a_hi, a_lo, a_f32, cand_parent, cand_gparent);
+                                                                  feat_norm, a_op, lay, a_f32, cand_parent, cand_gparent);
   else
     k_final_norm_mix<float><<<grid, kNormThreads, 0, s>>>(static_cast<const float*>(hidden), sh.B, T, sh.h, gamma, eps,
-                                                          cfg_scale, inv_temperature, feat, feat_norm, a_hi, a_lo, a_f32,
+                                                          cfg_scale, inv_temperature, feat, feat_norm, a_op, lay, a_f32,
                                                           cand_parent, cand_gparent);
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;

@@ -8,9 +8,10 @@
 // The projections run on the tensor-core GEMM in sliced mode (K cut into S slices, one output matrix
 // per slice); the row-wise kernels here add the S matrices while they do their own work, so no GEMM
 // waits for another CTA.  The residual stream x stays fp32; GEMM operands are written as a bf16 high
-// part plus a bf16 remainder.
+// part plus a bf16 remainder, in the staged layout the GEMM copies straight into shared memory.
 #include "cascade_internal.h"
 #include "gemm_tc.h"
+#include "operand.cuh"
 
 namespace {
 
@@ -29,17 +30,6 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 __device__ __forceinline__ float elem_to_float(const float* p, size_t i) { return p[i]; }
 __device__ __forceinline__ float elem_to_float(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
 
-// writes one operand value: bf16 high part + remainder, or fp32
-__device__ __forceinline__ void put_operand(__nv_bfloat16* hi, __nv_bfloat16* lo, float* f32, size_t i, float a) {
-  if (hi != nullptr) {
-    const __nv_bfloat16 h = __float2bfloat16_rn(a);
-    hi[i] = h;
-    lo[i] = __float2bfloat16_rn(a - __bfloat162float(h));
-  } else {
-    f32[i] = a;
-  }
-}
-
 __device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
   const uint2 r = *reinterpret_cast<const uint2*>(p);
@@ -52,23 +42,25 @@ __device__ __forceinline__ void add4(float4& a, const float4 b) {
   a.z += b.z;
   a.w += b.w;
 }
-// four consecutive operand values
-__device__ __forceinline__ void put_operand4(__nv_bfloat16* hi, __nv_bfloat16* lo, float* f32, size_t i, const float4 a) {
-  if (hi != nullptr) {
+// four consecutive operand values of row m, columns k..k+3 (k a multiple of 4): fp32, or the bf16 pair in the
+// GEMM's staged layout
+__device__ __forceinline__ void put_operand4(__nv_bfloat16* op, const OperandLayout& lay, float* f32, int K, int m, int k,
+                                             const float4 a) {
+  if (op != nullptr) {
     const float v[4] = {a.x, a.y, a.z, a.w};
     uint32_t h[2], l[2];
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * k]), h1 = __float2bfloat16_rn(v[2 * k + 1]);
-      const __nv_bfloat16 l0 = __float2bfloat16_rn(v[2 * k] - __bfloat162float(h0));
-      const __nv_bfloat16 l1 = __float2bfloat16_rn(v[2 * k + 1] - __bfloat162float(h1));
-      h[k] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-      l[k] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    for (int i = 0; i < 2; ++i) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * i]), h1 = __float2bfloat16_rn(v[2 * i + 1]);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(v[2 * i] - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(v[2 * i + 1] - __bfloat162float(h1));
+      h[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      l[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
     }
-    *reinterpret_cast<uint2*>(hi + i) = make_uint2(h[0], h[1]);
-    *reinterpret_cast<uint2*>(lo + i) = make_uint2(l[0], l[1]);
+    *reinterpret_cast<uint2*>(op + operand_index(lay, m, k, 0)) = make_uint2(h[0], h[1]);
+    *reinterpret_cast<uint2*>(op + operand_index(lay, m, k, 1)) = make_uint2(l[0], l[1]);
   } else {
-    *reinterpret_cast<float4*>(f32 + i) = a;
+    *reinterpret_cast<float4*>(f32 + (size_t)m * K + k) = a;
   }
 }
 
@@ -84,8 +76,8 @@ __global__ void __launch_bounds__(kRowThreads) k_resid_norm(float* __restrict__ 
                                                             const int32_t* __restrict__ tok,
                                                             const float* __restrict__ slices, int n_slices,
                                                             long long slice_stride, const float* __restrict__ gamma,
-                                                            float eps, __nv_bfloat16* __restrict__ a_hi,
-                                                            __nv_bfloat16* __restrict__ a_lo, float* __restrict__ a_f32,
+                                                            float eps, __nv_bfloat16* __restrict__ a_op,
+                                                            const OperandLayout lay, float* __restrict__ a_f32,
                                                             float* __restrict__ x_copy) {
   __shared__ float red[kRowThreads / 32];
   const int m = blockIdx.x;
@@ -126,7 +118,7 @@ __global__ void __launch_bounds__(kRowThreads) k_resid_norm(float* __restrict__ 
   const float rs = rsqrtf(ss / h + eps);
   auto emit = [&](int c, const float4 v) {
     const float4 g = load4(gamma + 4 * c);
-    put_operand4(a_hi, a_lo, a_f32, (size_t)m * h + 4 * c, make_float4(v.x * rs * g.x, v.y * rs * g.y, v.z * rs * g.z, v.w * rs * g.w));
+    put_operand4(a_op, lay, a_f32, h, m, 4 * c, make_float4(v.x * rs * g.x, v.y * rs * g.y, v.z * rs * g.z, v.w * rs * g.w));
   };
 #pragma unroll
   for (int k = 0; k < kRowChunks; ++k) {
@@ -200,8 +192,8 @@ __global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restr
 // ffn is a multiple of 4.
 __global__ void __launch_bounds__(kRowThreads) k_swiglu(const float* __restrict__ slices, int n_slices,
                                                         long long slice_stride, int ffn,
-                                                        __nv_bfloat16* __restrict__ a_hi,
-                                                        __nv_bfloat16* __restrict__ a_lo, float* __restrict__ a_f32) {
+                                                        __nv_bfloat16* __restrict__ a_op, const OperandLayout lay,
+                                                        float* __restrict__ a_f32) {
   const size_t m = blockIdx.y;
   for (int c = blockIdx.x * kRowThreads + threadIdx.x; c < ffn / 4; c += gridDim.x * kRowThreads) {
     float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
@@ -210,7 +202,7 @@ __global__ void __launch_bounds__(kRowThreads) k_swiglu(const float* __restrict_
       add4(g, load4(row + 4 * c));
       add4(u, load4(row + ffn + 4 * c));
     }
-    put_operand4(a_hi, a_lo, a_f32, m * ffn + 4 * c,
+    put_operand4(a_op, lay, a_f32, ffn, (int)m, 4 * c,
                  make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
                              g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w));
   }
@@ -250,10 +242,9 @@ int project(cascade_ctx* ctx, const void* W, int N, int K, int M, bool operand_i
     e.splits = S;
     e.slice_stride = pr->slice_stride;
     if ((long long)S * M * N > ctx->gemm_out_floats) return CASCADE_ERR_WORKSPACE;
-    if (operand_is_attn)  // the attention wrote its output as a bf16 high part plus remainder
-      return launch_gemm_tc(ctx, (const __nv_bfloat16*)W, N, K, (const __nv_bfloat16*)ctx->attn_out, ctx->attn_lo_offset, M,
-                            e, kernel_id, s);
-    return launch_gemm_tc(ctx, (const __nv_bfloat16*)W, N, K, ctx->act_hi, ctx->act_lo_offset, M, e, kernel_id, s);
+    // the operand is already in the GEMM's staged layout (the attention writes its output that way too)
+    return launch_gemm_tc(ctx, (const __nv_bfloat16*)W, N, K,
+                          operand_is_attn ? (const __nv_bfloat16*)ctx->attn_out : ctx->act, M, e, kernel_id, s);
   }
   pr->n_slices = 1;
   dim3 grid(cascade_detail::ceil_div(N, 8), cascade_detail::ceil_div(M, 8));
@@ -275,8 +266,8 @@ int resid_norm(cascade_ctx* ctx, int T, const void* embed, const int32_t* tok, c
   KernelScope ks(ctx, kernel_id, s);
   k_resid_norm<E><<<M, kRowThreads, 0, s>>>(ctx->x, sh.B, T, sh.h, (const E*)embed, tok, ctx->gemm_out,
                                             pr ? pr->n_slices : 0, pr ? pr->slice_stride : 0, gamma, eps,
-                                            bf16 ? ctx->act_hi : nullptr, bf16 ? ctx->act_hi + ctx->act_lo_offset : nullptr,
-                                            bf16 ? nullptr : ctx->act_f32, x_copy);
+                                            bf16 ? ctx->act : nullptr, operand_layout(M, sh.h), bf16 ? nullptr : ctx->act_f32,
+                                            x_copy);
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }
@@ -318,8 +309,7 @@ int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step*
       CASCADE_TRY(launch_tree_attn_bf16(ctx, tree, (const __nv_bfloat16*)ctx->q_rot, (const __nv_bfloat16*)L.k_prefix,
                                         (const __nv_bfloat16*)L.v_prefix, st->prefix_cap, st->prefix_len,
                                         (const __nv_bfloat16*)k_rot, (const __nv_bfloat16*)v_rot,
-                                        (__nv_bfloat16*)ctx->attn_out,
-                                        (__nv_bfloat16*)ctx->attn_out + ctx->attn_lo_offset, st->softmax_scale, s));
+                                        (__nv_bfloat16*)ctx->attn_out, true, st->softmax_scale, s));
     else
       CASCADE_TRY(launch_tree_attn_f32(ctx, tree, (const float*)ctx->q_rot, (const float*)L.k_prefix,
                                        (const float*)L.v_prefix, st->prefix_cap, st->prefix_len, (const float*)k_rot,
@@ -334,8 +324,8 @@ int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step*
       const bool bf16 = sh.dtype == CASCADE_BF16;
       KernelScope ks(ctx, K_SWIGLU, s);
       k_swiglu<<<dim3(cascade_detail::ceil_div(sh.ffn / 4, kRowThreads), M), kRowThreads, 0, s>>>(
-          ctx->gemm_out, pr.n_slices, pr.slice_stride, sh.ffn, bf16 ? ctx->act_hi : nullptr,
-          bf16 ? ctx->act_hi + ctx->act_lo_offset : nullptr, bf16 ? nullptr : ctx->act_f32);
+          ctx->gemm_out, pr.n_slices, pr.slice_stride, sh.ffn, bf16 ? ctx->act : nullptr, operand_layout(M, sh.ffn),
+          bf16 ? nullptr : ctx->act_f32);
     }
     CASCADE_CUDA_TRY(cudaGetLastError());
     CASCADE_TRY(project(ctx, L.w_down, sh.h, sh.ffn, M, false, K_GEMM_DOWN, &pr, s));
