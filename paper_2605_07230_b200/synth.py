@@ -341,18 +341,29 @@ def uniforms(rng, B: int, T: int) -> np.ndarray:
     return rng.random((B, T), dtype=np.float32)
 
 
-def layer_step_inputs(w: Workload, rng, parent, n_layers: int = 1):
+def layer_step_inputs(w: Workload, rng, parent, n_layers: int = 1, out_scale=None):
     """Inputs of a verification step that runs through decoder layers: the clustered codebook as token
     embedding and (tied) LM head, `n_layers` sets of N(0, 0.02) layer weights, an N(0,1) prefix KV cache
     per layer (independent for the cond and uncond rows), stand-in drafter tokens and probabilities,
-    uniforms.  Everything is returned in the values the workload's element type can hold."""
+    uniforms.  Everything is returned in the values the workload's element type can hold.
+
+    out_scale = (s_o, s_down) multiplies the output projection and the MLP down projection.  With plain
+    N(0, 0.02) matrices of these widths one layer's update is ~100x the norm of the token embedding, the
+    final hidden state forgets its token and no draft is ever accepted; the default for the 7B-shaped
+    workloads, (0.05, 0.005), keeps the update at about 0.6x the embedding norm (as in a trained model,
+    where a layer nudges the residual stream), so that acceptance and relaxation both take part.  The
+    fp32 toy workload keeps the plain weights its definition names."""
     T = len(parent)
     R, H, D, P = 2 * w.B, w.n_heads, w.head_dim, w.prefix_len
     E = quantize(clustered_codebook(rng, w.V, w.h, w.n_clusters, w.sigma), w.dtype)
+    if out_scale is None:
+        out_scale = (1.0, 1.0) if w.name == "toy" else (0.05, 0.005)
     layers = []
     caches = []
     for _ in range(n_layers):
         lw = layer_weights(rng, w.h, H, D, w.ffn)
+        lw.wo = lw.wo * np.float32(out_scale[0])
+        lw.w_down = lw.w_down * np.float32(out_scale[1])
         for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"):
             setattr(lw, name, quantize(getattr(lw, name), w.dtype))
         layers.append(lw)

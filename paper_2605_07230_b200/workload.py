@@ -138,7 +138,8 @@ class LayerWorkload:
     rotates through them so that a step never finds its operands in the L2)."""
 
     def __init__(self, w: synth.Workload, n_layers: int = 1, device="cuda:0", n_sets: int = 1,
-                 keep_logits: bool = False, select_mode: int = cb.SELECT_LONGEST, flags: int = cb.USE_I | cb.USE_C):
+                 keep_logits: bool = False, select_mode: int = cb.SELECT_LONGEST, flags: int = cb.USE_I | cb.USE_C,
+                 host: dict | None = None):
         self.w, self.device, self.n_layers = w, device, n_layers
         self.parent = w.parent()
         T = self.T = len(self.parent)
@@ -147,7 +148,7 @@ class LayerWorkload:
         self.tree = cb.Tree(self.ctx, self.parent)
         self.params = cb.Params(w.tau_pos, w.tau_seq, w.tvd_budget, flags)
         rng = np.random.default_rng(w.seed)
-        self.host = synth.layer_step_inputs(w, rng, self.parent, n_layers)
+        self.host = host if host is not None else synth.layer_step_inputs(w, rng, self.parent, n_layers)
         self.sets = [self._make_set(self.host if i == 0 else self._fresh_step(i), keep_logits, select_mode)
                      for i in range(n_sets)]
 

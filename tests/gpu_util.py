@@ -68,3 +68,33 @@ def compare_decisions(parent, oracle_rows, accept_gpu, path_nodes_gpu, path_len_
             assert np.all(path_nodes_gpu[b][alpha + 1:] == -1)
             stats["paths_compared"] += 1
     return stats
+
+
+def target_sampled_drafts(w, host, parent, rng, temperature=1.5):
+    """Draft tokens drawn level by level from the TARGET's own softened distribution (the toy workload's
+    definition): children of node j are sampled without replacement from softmax(logits[j] / temperature),
+    best first, with that softened probability as the drafter's p.  Needs the checker's forward pass once
+    per level (a row's logits depend only on the tokens of its ancestors), so it is only for small cases."""
+    T = len(parent)
+    kids = O.children_of(parent)
+    depth = O.tree_depth(parent)
+    tok = host["tok"].copy()
+    p = np.ones_like(host["draft_p"])
+    for level in range(int(depth.max())):
+        out = O.verify_step(host["embed"], host["layers"], host["gamma_final"], host["w_head"], tok, parent,
+                            host["k_prefix"], host["v_prefix"], host["prefix_len"], p, host["uniforms"], w.n_heads,
+                            w.head_dim, w.eps, w.rope_base, w.cfg_scale, 1.0, w.tau_pos, w.tau_seq, w.tvd_budget,
+                            kv_bf16=w.dtype == "bf16")
+        logits = out["head"]["logits"]
+        for b in range(w.B):
+            for j in range(T):
+                if depth[j] != level or not kids[j]:
+                    continue
+                soft = O.softmax(logits[b, j] / temperature)
+                g = np.log(np.maximum(soft, 1e-300)) - np.log(-np.log(rng.random(len(soft))))
+                pick = np.argsort(-g)[: len(kids[j])]
+                pick = pick[np.argsort(-soft[pick], kind="stable")]
+                for kid, t in zip(kids[j], pick):
+                    tok[b, kid] = t
+                    p[b, kid] = soft[t]
+    return tok.astype(np.int32), p.astype(np.float32)

@@ -28,7 +28,13 @@ def oracle_step(wl, host):
 ])
 def test_step_through_layers(name, over, n_layers):
     w = synth.workload(name, **over)
-    wl = LayerWorkload(w, n_layers=n_layers, keep_logits=True)
+    host = None
+    if name == "toy":
+        # config 1: plain N(0, 0.02) weights and draft tokens sampled from the target's softmax at T = 1.5
+        parent = w.parent()
+        host = synth.layer_step_inputs(w, np.random.default_rng(w.seed), parent, n_layers)
+        host["tok"], host["draft_p"] = G.target_sampled_drafts(w, host, parent, np.random.default_rng(7))
+    wl = LayerWorkload(w, n_layers=n_layers, keep_logits=True, host=host)
     s = wl.run(0)
     torch.cuda.synchronize()
     wl.ctx.check()
@@ -50,8 +56,10 @@ def test_step_through_layers(name, over, n_layers):
                              s.host["uniforms"][b], w.tau_pos, w.tau_seq, w.tvd_budget) for b in range(w.B)]
     G.compare_decisions(wl.parent, rows, s.out["accept"].cpu().numpy(), s.out["path_nodes"].cpu().numpy(),
                         s.out["path_len"].cpu().numpy(), cb.SELECT_LONGEST)
+    accepted = int(s.out["accept"].cpu().numpy().sum()) - w.B
+    assert accepted > 0                      # the workload is not degenerate: some drafts are accepted
     print(f"{name} x{n_layers}: hidden max-abs {hid_err:.2e}, logits max-abs {logit_err:.2e}, "
-          f"{wl.ctx.last_launch_count} kernels")
+          f"{wl.ctx.last_launch_count} kernels, {accepted} drafts accepted, path lengths {s.out['path_len'].cpu().tolist()}")
     wl.close()
 
 
