@@ -42,6 +42,7 @@ extern "C" {
 #define CASCADE_ERR_UNSUPPORTED_SHAPE (-4) /* shape outside what the kernels handle (see cascade_shape) */
 #define CASCADE_ERR_CUDA (-5)              /* a CUDA runtime / driver call failed                      */
 #define CASCADE_ERR_TIMEOUT (-6)           /* a bounded device-side wait gave up (see cascade_check)   */
+#define CASCADE_ERR_OVERFLOW (-7)          /* cascade_kv_append: a cache has no room (see cascade_check) */
 
 /* ---- enums ------------------------------------------------------------------------------------- */
 #define CASCADE_F32 0
@@ -100,7 +101,7 @@ int cascade_destroy(cascade_ctx* ctx);
 int64_t cascade_workspace_bytes(const cascade_ctx* ctx);
 
 /* Reads the context's device-side error word (set when a bounded wait inside a kernel ran out) after
- * synchronising `stream`.  Returns CASCADE_OK, CASCADE_ERR_TIMEOUT or CASCADE_ERR_CUDA, and clears
+ * synchronising `stream`.  Returns CASCADE_OK, CASCADE_ERR_TIMEOUT, CASCADE_ERR_OVERFLOW or CASCADE_ERR_CUDA, and clears
  * the word. */
 int cascade_check(cascade_ctx* ctx, void* stream);
 
@@ -294,6 +295,33 @@ int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const c
                              const int32_t* tok_host, const float* draft_p_host, const float* uniforms_host,
                              uint8_t* accept_host, int32_t* path_nodes_host, int32_t* path_len_host,
                              void* stream);
+
+/* ---- between two steps of a decode loop --------------------------------------------------------- */
+/* The token after the accepted path: Algorithm 1's last step (the next token is drawn from the target
+ * distribution with the rejected proposals removed; from the target distribution itself after a fully
+ * accepted draft), which Algorithm 2 leaves out.  For prompt b, end = last node of its path; the tokens of
+ * end's children (all rejected, whichever selection mode chose the path) get probability zero, the rest of
+ * softmax(logits[b, end, :]) is renormalised, and token_out[b] is the inverse-CDF sample at u_bonus[b]:
+ * the first v whose cumulative weight exceeds u_bonus[b] * (remaining weight).
+ *   logits [B,T,V] float (as stored by cascade_lm_head_cfg / cascade_verify_step); tok [B,T] int32;
+ *   path_nodes [B,depth+1], path_len [B] from cascade_select_path; u_bonus [B] float in [0,1);
+ *   token_out [B] int32; mass_out [B] float or NULL: remaining probability mass after the removal. */
+int cascade_bonus_token(cascade_ctx* ctx, const cascade_tree* tree, const float* logits, const int32_t* tok,
+                        const int32_t* path_nodes, const int32_t* path_len, const float* u_bonus, int32_t* token_out,
+                        float* mass_out, void* stream);
+
+/* Appends the keys / values of the accepted path's tree rows (root row first: the pending token, then the
+ * accepted drafts) to the caches of n_layers layers, for both CFG rows of every prompt, at positions
+ * prefix_len[r] .. prefix_len[r] + path_len[b], and adds path_len[b] + 1 to prefix_len[r] (device array,
+ * updated in place).  The tree rows were rotated at exactly these positions by cascade_verify_step.
+ *   layers: HOST array of n_layers structs; only k_prefix / v_prefix are read, and those caches
+ *           ([R, prefix_cap, Hkv, D] elem) are WRITTEN here although the struct declares them const.
+ *   k_tree, v_tree [n_layers,R,T,Hkv,D] elem: cascade_step.k_tree_out / v_tree_out of the step.
+ * A path that does not fit into prefix_cap is not appended and raises CASCADE_ERR_OVERFLOW at the next
+ * cascade_check.  n_layers <= 64. */
+int cascade_kv_append(cascade_ctx* ctx, const cascade_tree* tree, int32_t n_layers, const cascade_layer* layers,
+                      const void* k_tree, const void* v_tree, const int32_t* path_nodes, const int32_t* path_len,
+                      int32_t prefix_cap, int32_t* prefix_len, void* stream);
 
 /* ---- acceptance without any device allocation --------------------------------------------------- */
 /* The paper has no counterpart to this entry point; it exists for deployment.  Some callers of this

@@ -360,6 +360,37 @@ def select_path(accept, parent, tvd_out=None, mode=SELECT_LONGEST):
     return path, int(depth[end]), tvd_used
 
 
+def bonus_token(logits_row, rejected_tokens, u):
+    """The token that follows the accepted path (Algorithm 1, last step: after a rejection the next token is
+    drawn from the target distribution with the rejected proposals removed; after a fully accepted path it is
+    drawn from the target distribution itself).  Algorithm 2 leaves this step out; the reading here: the
+    children of the path's end node were all rejected, their (distinct) tokens get probability zero, the rest
+    of softmax(logits_row) is renormalised, and the token is the inverse-CDF sample at u in [0,1):
+    the first v with cumsum(prob)[v] > u * total.  Returns (token, total = remaining mass)."""
+    g = softmax(np.asarray(logits_row, np.float64))
+    g = g.copy()
+    for t in set(int(x) for x in rejected_tokens):
+        g[t] = 0.0
+    total = float(g.sum())
+    c = np.cumsum(g)
+    v = int(np.searchsorted(c, float(u) * total, side="right"))
+    return min(v, len(g) - 1), total
+
+
+def append_path_kv(k_cache, v_cache, prefix_len, k_tree, v_tree, path, B):
+    """Cache update after a step: the tree rows on the accepted path (root first) are appended, in path
+    order, to both CFG rows' caches of one layer.  k_cache/v_cache [2B,cap,H,D] are modified in place;
+    returns the new prefix lengths."""
+    new_len = np.array(prefix_len, np.int64).copy()
+    for b, nodes in enumerate(path):
+        for r in (b, B + b):
+            for i, node in enumerate(nodes):
+                k_cache[r, prefix_len[r] + i] = k_tree[r, node]
+                v_cache[r, prefix_len[r] + i] = v_tree[r, node]
+            new_len[r] = prefix_len[r] + len(nodes)
+    return new_len
+
+
 # ------------------------------------------------------------------------------------------------
 # support: the rest of one decoder layer (architecture from the workload definition, not the paper)
 # ------------------------------------------------------------------------------------------------

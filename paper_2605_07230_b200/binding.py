@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcascade.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_TREE, ERR_WORKSPACE, ERR_UNSUPPORTED_SHAPE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
+ERR_OVERFLOW = -7
 F32, BF16 = 0, 1
 USE_I, USE_C, CONV_DIST_SELF = 1, 2, 4
 SELECT_LONGEST, SELECT_FIRST_ACCEPT = 0, 1
@@ -27,7 +28,7 @@ EXPORTS = [
     "cascade_strerror", "cascade_timing_enable", "cascade_timing_read", "cascade_kernel_name", "cascade_tree_create", "cascade_tree_destroy", "cascade_tree_rows", "cascade_tree_depth",
     "cascade_tree_num_pairs", "cascade_tree_pairs", "cascade_tree_attn", "cascade_lm_head_cfg",
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
-    "cascade_verify_step_host", "cascade_accept_static",
+    "cascade_verify_step_host", "cascade_accept_static", "cascade_bonus_token", "cascade_kv_append",
 ]
 
 
@@ -99,6 +100,8 @@ def lib() -> C.CDLL:
         L.cascade_verify_step_host.argtypes = [vp, vp, C.POINTER(Step), vp, vp, vp, vp, vp, vp, vp]
         L.cascade_accept_static.argtypes = [C.c_int32, C.c_int32, vp, vp, C.c_int32, vp, vp, vp, vp, vp, vp, vp,
                                             C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.cascade_bonus_token.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.cascade_kv_append.argtypes = [vp, vp, C.c_int32, C.POINTER(Layer), vp, vp, vp, vp, C.c_int32, vp, vp]
         _lib = L
     return _lib
 
@@ -292,3 +295,14 @@ def cascade_accept_static(B, parent, feat, feat_dim, feat_norm, row_lse, cand_pa
                                        _ptr(uniforms), C.byref(params), select_mode, _ptr(accept), _ptr(q_relaxed),
                                        _ptr(tvd_out), _ptr(near_count), _ptr(path_nodes), _ptr(path_len),
                                        _ptr(tvd_used), _stream()))
+
+
+def cascade_bonus_token(ctx, tree, logits, tok, path_nodes, path_len, u_bonus, token_out, mass_out=None):
+    _check(lib().cascade_bonus_token(ctx.handle, tree.handle, _ptr(logits), _ptr(tok), _ptr(path_nodes),
+                                     _ptr(path_len), _ptr(u_bonus), _ptr(token_out), _ptr(mass_out), _stream()))
+
+
+def cascade_kv_append(ctx, tree, step: Step, k_tree, v_tree, path_nodes, path_len, prefix_cap, prefix_len):
+    """Appends the accepted path's rows to the caches named in `step.layers` (a Step made by make_step)."""
+    _check(lib().cascade_kv_append(ctx.handle, tree.handle, step.n_layers, step.layers, _ptr(k_tree), _ptr(v_tree),
+                                   _ptr(path_nodes), _ptr(path_len), prefix_cap, _ptr(prefix_len), _stream()))

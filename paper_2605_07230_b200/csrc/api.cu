@@ -138,6 +138,7 @@ const char* cascade_strerror(int status) {
     case CASCADE_ERR_UNSUPPORTED_SHAPE: return "shape not supported by the kernels";
     case CASCADE_ERR_CUDA: return "a CUDA call failed";
     case CASCADE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case CASCADE_ERR_OVERFLOW: return "a KV cache has no room for the accepted path";
     default: return "unknown status";
   }
 }
@@ -146,7 +147,7 @@ const char* cascade_kernel_name(int32_t id) {
   static const char* names[] = {"tree_attn", "tree_attn_f32", "final_norm_mix", "gemm_head",
                                 "head_f32", "row_stats", "row_lse", "similarity", "accept", "tail", "select_path",
                                 "embed_norm", "gemm_qkv", "rope_split", "gemm_o", "resid_norm", "gemm_gate_up",
-                                "swiglu", "gemm_down", "gemm_f32", "resid_add"};
+                                "swiglu", "gemm_down", "gemm_f32", "resid_add", "kv_append", "bonus_token"};
   static_assert(sizeof(names) / sizeof(names[0]) == K_KERNEL_ID_END, "one name per kernel id");
   if (id < 0 || id >= K_KERNEL_ID_END) return nullptr;
   return names[id];
@@ -240,7 +241,7 @@ int cascade_check(cascade_ctx* ctx, void* stream) {
   if (word != 0) {
     CASCADE_CUDA_TRY(cudaMemsetAsync(ctx->dev_error, 0, sizeof(int), s));
     CASCADE_CUDA_TRY(cudaStreamSynchronize(s));
-    return CASCADE_ERR_TIMEOUT;
+    return (word & CASCADE_DEV_ERR_WAIT) ? CASCADE_ERR_TIMEOUT : CASCADE_ERR_OVERFLOW;
   }
   return CASCADE_OK;
 }

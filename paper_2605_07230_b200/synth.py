@@ -206,6 +206,7 @@ def cluster_drafter(
     n_clusters: int,
     stay: float = 0.75,
     sharp: float = 1.6,
+    roots=None,
 ):
     """Target-free stand-in for a trained drafter.
 
@@ -214,6 +215,7 @@ def cluster_drafter(
     random per-code weight raised to `sharp`; the children of one parent are drawn from it without
     replacement, best first.  Returns tok[B,T] (row 0 = the pending root token) and draft_p[B,T]
     (probability the stand-in assigned to each drafted token under its parent's context; row 0 = 1).
+    `roots` [B] fixes the root tokens (a decode loop's pending tokens) instead of drawing them.
     """
     T = len(parent)
     per = V // n_clusters
@@ -223,7 +225,7 @@ def cluster_drafter(
     for j in range(1, T):
         children[parent[j]].append(j)
     for b in range(B):
-        tok[b, 0] = int(rng.integers(0, V))
+        tok[b, 0] = int(rng.integers(0, V)) if roots is None else int(roots[b])
         for j in range(T):
             kids = children[j]
             if not kids:

@@ -213,3 +213,84 @@ class LayerWorkload:
         e = 2 if w.dtype == "bf16" else 4
         hd = w.n_heads * w.head_dim
         return {"layer": (3 * hd * w.h + w.h * hd + 3 * w.ffn * w.h) * e * self.n_layers, "lm_head": w.V * w.h * e}
+
+
+class DecodeLoop:
+    """A speculative decode loop around the verification step (the last workload of the set: many layers,
+    the caches grow by the accepted tokens every step).  Per step: the stand-in drafter proposes a tree
+    below each prompt's pending token (host), the library verifies it (cascade_verify_step), draws the
+    token after the accepted path (cascade_bonus_token) and appends the accepted rows to every layer's
+    cache (cascade_kv_append); the host reads back the path and the new pending token.  Data movement and
+    argument marshalling only."""
+
+    def __init__(self, w: synth.Workload, n_layers: int, max_steps: int, device="cuda:0", seed: int = 0,
+                 select_mode: int = cb.SELECT_LONGEST):
+        self.w, self.n_layers, self.device = w, n_layers, device
+        self.parent = w.parent()
+        T = self.T = len(self.parent)
+        depth = int(synth.tree_depth(self.parent).max())
+        self.cap = w.prefix_len + max_steps * (depth + 1)
+        B, R = w.B, 2 * w.B
+        self.ctx = cb.Context(cb.BF16 if w.dtype == "bf16" else cb.F32, B, T, self.cap, w.h, w.n_heads, w.n_heads,
+                              w.head_dim, w.V, w.ffn)
+        self.tree = cb.Tree(self.ctx, self.parent)
+        self.params = cb.Params(w.tau_pos, w.tau_seq, w.tvd_budget, cb.USE_I | cb.USE_C)
+        rng = np.random.default_rng(w.seed)
+        host = synth.layer_step_inputs(w, rng, self.parent, n_layers)
+        # caches with room for the whole run; the first prefix_len rows hold the seeded prompt cache
+        for li in range(n_layers):
+            for name in ("k_prefix", "v_prefix"):
+                full = np.zeros((R, self.cap, w.n_heads, w.head_dim), np.float32)
+                full[:, :w.prefix_len] = host[name][li]
+                host[name][li] = full
+        self.host = host
+        self.rng = np.random.default_rng(seed)
+        self.roots = host["tok"][:, 0].copy()
+        self.prefix_len_host = host["prefix_len"].astype(np.int64).copy()
+        wl = LayerWorkload.__new__(LayerWorkload)   # reuse its buffer set-up on this context
+        wl.w, wl.device, wl.n_layers, wl.parent, wl.T, wl.ctx, wl.tree, wl.params = (w, device, n_layers, self.parent, T,
+                                                                                     self.ctx, self.tree, self.params)
+        w_cap = synth.Workload(**{**w.__dict__, "prefix_len": self.cap})
+        wl.w = w_cap
+        self.set = wl._make_set(host, True, select_mode)
+        self.set.step.prefix_cap = self.cap
+        self.u_bonus = torch.zeros(B, device=device)
+        self.bonus = torch.zeros(B, dtype=torch.int32, device=device)
+        self.mass = torch.zeros(B, device=device)
+        self.emitted = [[] for _ in range(B)]
+
+    def draft(self):
+        """Next tree of the stand-in drafter below the pending tokens, plus this step's uniforms."""
+        w = self.w
+        tok, p = synth.cluster_drafter(self.rng, self.parent, w.B, w.V, w.n_clusters, roots=self.roots)
+        u = synth.uniforms(self.rng, w.B, self.T)
+        ub = self.rng.random(w.B, dtype=np.float32)
+        return tok, p, u, ub
+
+    def step(self, drafted=None):
+        tok, p, u, ub = drafted if drafted is not None else self.draft()
+        d, o = self.set.dev, self.set.out
+        d["tok"].copy_(torch.from_numpy(tok))
+        d["draft_p"].copy_(torch.from_numpy(p))
+        d["uniforms"].copy_(torch.from_numpy(u))
+        self.u_bonus.copy_(torch.from_numpy(ub))
+        cb.cascade_verify_step(self.ctx, self.tree, self.set.step)
+        cb.cascade_bonus_token(self.ctx, self.tree, o["logits"], d["tok"], o["path_nodes"], o["path_len"], self.u_bonus,
+                               self.bonus, self.mass)
+        cb.cascade_kv_append(self.ctx, self.tree, self.set.step, o["k_tree_out"], o["v_tree_out"], o["path_nodes"],
+                             o["path_len"], self.cap, d["prefix_len"])
+        plen = o["path_len"].cpu().numpy()
+        nodes = o["path_nodes"].cpu().numpy()
+        bonus = self.bonus.cpu().numpy()
+        self.ctx.check()
+        for b in range(self.w.B):
+            path = nodes[b][: plen[b] + 1]
+            self.emitted[b].extend(int(tok[b, j]) for j in path[1:])
+            self.emitted[b].append(int(bonus[b]))
+            self.prefix_len_host[[b, self.w.B + b]] += plen[b] + 1
+        self.roots = bonus.copy()
+        return dict(tok=tok, draft_p=p, uniforms=u, u_bonus=ub, path_len=plen, path_nodes=nodes, bonus=bonus)
+
+    def close(self):
+        self.tree.close()
+        self.ctx.close()

@@ -1,0 +1,93 @@
+"""GPU parity of a short speculative decode loop (verification step through several layers, bonus token,
+cache append) against the checker.  The checker follows the device's decisions from step to step
+(its own caches, its own arithmetic), so that a near-tie in one step cannot derail the comparison of
+the next."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cascade_oracle as O
+from paper_2605_07230_b200 import binding as cb
+from paper_2605_07230_b200 import synth
+from paper_2605_07230_b200.workload import DecodeLoop
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("over,n_layers,steps", [
+    (dict(B=2, tree="topk32", prefix_len=40), 2, 3),
+    (dict(B=1, tree="topk60", prefix_len=130), 3, 2),
+])
+def test_decode_loop(over, n_layers, steps):
+    w = synth.workload("mini", **over)
+    loop = DecodeLoop(w, n_layers, max_steps=steps, seed=11)
+    B, parent = w.B, loop.parent
+    h = loop.host
+    k_cache = [np.array(x, np.float64) for x in h["k_prefix"]]
+    v_cache = [np.array(x, np.float64) for x in h["v_prefix"]]
+    plen = h["prefix_len"].astype(np.int64).copy()
+    total_accepted = 0
+    for it in range(steps):
+        drafted = loop.draft()
+        tok, p, u, ub = drafted
+        ref = O.verify_step(h["embed"], h["layers"], h["gamma_final"], h["w_head"], tok, parent, k_cache, v_cache, plen,
+                            p, u, w.n_heads, w.head_dim, w.eps, w.rope_base, w.cfg_scale, 1.0, w.tau_pos, w.tau_seq,
+                            w.tvd_budget)
+        res = loop.step(drafted)
+        torch.cuda.synchronize()
+        o = loop.set.out
+        logits = o["logits"].cpu().numpy()
+        assert np.abs(logits - ref["head"]["logits"]).max() < 3e-2
+        feat = o["feat"].cpu().numpy().astype(np.float64)
+        rows = [O.relaxed_accept(feat[b], logits[b], tok[b], parent, p[b], u[b], w.tau_pos, w.tau_seq, w.tvd_budget)
+                for b in range(B)]
+        G.compare_decisions(parent, rows, o["accept"].cpu().numpy(), res["path_nodes"], res["path_len"], cb.SELECT_LONGEST)
+        kids = O.children_of(parent)
+        paths = []
+        for b in range(B):
+            path = [int(x) for x in res["path_nodes"][b][: res["path_len"][b] + 1]]
+            paths.append(path)
+            end = path[-1]
+            want, mass = O.bonus_token(logits[b, end], [tok[b, c] for c in kids[end]], ub[b])
+            if want != res["bonus"][b]:
+                # only a draw that lands on a boundary of the cumulative distribution may differ, by one place
+                g = O.softmax(logits[b, end].astype(np.float64))
+                for c in kids[end]:
+                    g[tok[b, c]] = 0
+                c = np.cumsum(g)
+                assert abs(c[min(want, res["bonus"][b])] - ub[b] * g.sum()) < 1e-5
+            assert abs(float(loop.mass[b]) - mass) < 1e-4
+            total_accepted += len(path) - 1
+        # cache append: exactly the rotated tree rows of the path, at the old prefix lengths, in every layer
+        k_out = o["k_tree_out"].float().cpu().numpy()
+        v_out = o["v_tree_out"].float().cpu().numpy()
+        new_len = loop.set.dev["prefix_len"].cpu().numpy()
+        for li in range(n_layers):
+            kc = loop.set.dev["layers"][li]["k_prefix"].float().cpu().numpy()
+            vc = loop.set.dev["layers"][li]["v_prefix"].float().cpu().numpy()
+            for b in range(B):
+                for r in (b, B + b):
+                    n = len(paths[b])
+                    assert np.array_equal(kc[r, plen[r]:plen[r] + n], k_out[li, r, paths[b]])
+                    assert np.array_equal(vc[r, plen[r]:plen[r] + n], v_out[li, r, paths[b]])
+                    assert new_len[r] == plen[r] + n
+            # the checker's caches take its own rows for the same path
+            q_ref, k_ref, v_ref = ref["attn_io"][li]
+            O.append_path_kv(k_cache[li], v_cache[li], plen, k_ref, v_ref, paths, B)
+        plen = np.array([plen[r] + len(paths[r % B]) for r in range(2 * B)])
+        assert np.array_equal(plen, loop.prefix_len_host)
+    assert total_accepted > 0
+    assert all(len(e) >= steps for e in loop.emitted)
+    loop.close()
+
+
+def test_append_beyond_the_cache_is_refused_not_written():
+    w = synth.workload("mini", B=1, tree="topk16", prefix_len=40)
+    loop = DecodeLoop(w, 1, max_steps=1, seed=3)
+    loop.step()
+    with pytest.raises(cb.CascadeError) as e:   # the second step has no room left
+        loop.step()
+        loop.step()
+    assert e.value.status == cb.ERR_OVERFLOW
+    loop.close()

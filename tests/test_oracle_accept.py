@@ -339,3 +339,49 @@ def test_cosine_properties():
     cs, cc = O.similarity_scores(np.array([[1.0, 0], [1, 0], [0, 2], [1, 1]]), np.array([-1, 0, 0, 1]))
     assert set(cs) == {(1, 2), (2, 1)} and set(cc) == {(0, 1), (0, 2), (1, 3)}
     assert cs[(1, 2)] == 0 and abs(cc[(1, 3)] - 2 ** -0.5) < 1e-15
+
+
+# ---- bonus token (Algorithm 1's final draw) and cache append ---------------------------------------
+
+
+def test_bonus_token_is_the_inverse_cdf_sample_of_the_renormalised_target():
+    rng = np.random.default_rng(3)
+    logits = rng.normal(0, 2, 50)
+    g = np.exp(logits - logits.max())
+    g /= g.sum()
+    # nothing rejected: plain inverse CDF, checked against a brute-force scan
+    for u in [0.0, 0.1, 0.5, 0.999999]:
+        tok, total = O.bonus_token(logits, [], u)
+        acc, want = 0.0, None
+        for v in range(50):
+            acc += g[v]
+            if acc > u:
+                want = v
+                break
+        assert tok == want and abs(total - 1.0) < 1e-12
+    # rejected tokens can never come back, and the rest keeps its proportions
+    rejected = [int(np.argmax(g)), 7, 7]
+    counts = np.zeros(50)
+    us = (np.arange(20000) + 0.5) / 20000
+    for u in us:
+        tok, total = O.bonus_token(logits, rejected, u)
+        counts[tok] += 1
+    assert counts[rejected[0]] == 0 and counts[7] == 0
+    rest = g.copy()
+    rest[rejected] = 0
+    assert abs(total - rest.sum()) < 1e-12
+    assert np.abs(counts / len(us) - rest / rest.sum()).max() < 2e-4
+
+
+def test_append_path_kv_writes_the_path_rows_in_order_to_both_cfg_rows():
+    B, cap, H, D, T = 2, 12, 1, 2, 5
+    k = np.zeros((2 * B, cap, H, D))
+    v = np.zeros((2 * B, cap, H, D))
+    kt = np.arange(2 * B * T * H * D, dtype=float).reshape(2 * B, T, H, D)
+    vt = -kt
+    plen = np.array([3, 4, 5, 6])
+    new = O.append_path_kv(k, v, plen, kt, vt, [[0, 2, 4], [0]], B)
+    assert new.tolist() == [6, 5, 8, 7]
+    assert np.array_equal(k[0, 3:6], kt[0, [0, 2, 4]]) and np.array_equal(k[2, 5:8], kt[2, [0, 2, 4]])
+    assert np.array_equal(v[1, 4:5], vt[1, [0]]) and np.array_equal(v[3, 6:7], vt[3, [0]])
+    assert k[0, 6:].sum() == 0 and k[1, 5:].sum() == 0
