@@ -333,9 +333,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
             const int pi = e.parent[j];
             if (pi < 0) continue;
             const int gp = e.parent[pi];
+            // columns are activation rows relative to this row chunk; rows of other chunks are served by
+            // the CTAs that hold those chunks (-1: not here)
+            const int n_valid = min(NB, p.M - m0);
+            int cp = b * e.T + pi - m0, cg = gp >= 0 ? b * e.T + gp - m0 : -1;
+            if ((unsigned)cp >= (unsigned)n_valid) cp = -1;
+            if ((unsigned)cg >= (unsigned)n_valid) cg = -1;
+            if (cp < 0 && cg < 0) continue;
             const int pos = atomicAdd(&s_gather_n, 1);
-            if (pos < kGatherCap)
-              s_gather[pos] = make_int4((ln >> 5) * 33 + (ln & 31), b * e.T + pi - m0, gp >= 0 ? b * e.T + gp - m0 : -1, idx);
+            if (pos < kGatherCap) s_gather[pos] = make_int4((ln >> 5) * 33 + (ln & 31), cp, cg, idx);
           }
           ptx::named_bar_sync(1, 128);
           n_gather = s_gather_n;
@@ -425,7 +431,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
                 for (int i = eid; i < n_gather; i += 128) {
                   const int4 g = s_gather[i];
                   int col = g.y - cs;
-                  if ((unsigned)col < (unsigned)kStCols) e.cand_parent[g.w] = st[col * kStRow + g.x];
+                  if (g.y >= 0 && (unsigned)col < (unsigned)kStCols) e.cand_parent[g.w] = st[col * kStRow + g.x];
                   col = g.z - cs;
                   if (g.z >= 0 && (unsigned)col < (unsigned)kStCols) e.cand_gparent[g.w] = st[col * kStRow + g.x];
                 }
@@ -438,12 +444,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
                   const int pi = e.parent[j];
                   if (pi < 0) continue;
                   const int at = (ln >> 5) * 33 + (ln & 31);
-                  int col = b * e.T + pi - m0 - cs;
-                  if ((unsigned)col < (unsigned)kStCols) e.cand_parent[idx] = st[col * kStRow + at];
+                  const int n_valid = min(NB, p.M - m0);
+                  int row = b * e.T + pi - m0, col = row - cs;
+                  if ((unsigned)row < (unsigned)n_valid && (unsigned)col < (unsigned)kStCols)
+                    e.cand_parent[idx] = st[col * kStRow + at];
                   const int gp = e.parent[pi];
                   if (gp < 0) continue;
-                  col = b * e.T + gp - m0 - cs;
-                  if ((unsigned)col < (unsigned)kStCols) e.cand_gparent[idx] = st[col * kStRow + at];
+                  row = b * e.T + gp - m0;
+                  col = row - cs;
+                  if ((unsigned)row < (unsigned)n_valid && (unsigned)col < (unsigned)kStCols)
+                    e.cand_gparent[idx] = st[col * kStRow + at];
                 }
               }
             }
