@@ -213,7 +213,7 @@ def main():
     per_set = (w.V * w.h + 2 * 2 * w.B * (w.prefix_len + T) * hd) * 2 + layer_bytes
     n_sets = args.sets or max(2, int(np.ceil(3 * 126e6 / per_set)))
     if args.mode == "layer":
-        wl = LayerWorkload(w, n_layers=1, device=dev, n_sets=n_sets)
+        wl = LayerWorkload(w, n_layers=1, device=dev, n_sets=n_sets, want_hidden=False)
     else:
         wl = PiecesWorkload(w, device=dev, n_sets=n_sets)
     K, W = args.steps, max(args.warmup, 3)

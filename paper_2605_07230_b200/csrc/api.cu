@@ -395,7 +395,7 @@ static int lm_head_impl(cascade_ctx* ctx, const cascade_tree* tree, const void* 
                         float eps, const void* w_head, float cfg_scale, float temperature, const int32_t* tok,
                         float* logits_out, float* feat_out, float* feat_norm_out, float* row_lse_out,
                         float* cand_parent_out, float* cand_gparent_out, bool fold_lse, bool hidden_f32,
-                        cudaStream_t s) {
+                        const PendingAdd& add, cudaStream_t s) {
   if (ctx == nullptr || tree == nullptr || hidden == nullptr || rms_gamma == nullptr || w_head == nullptr)
     return CASCADE_ERR_INVALID_ARG;
   if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;
@@ -405,7 +405,7 @@ static int lm_head_impl(cascade_ctx* ctx, const cascade_tree* tree, const void* 
       !aligned16(rms_gamma))
     return CASCADE_ERR_INVALID_ARG;
   if (row_lse_out == nullptr) row_lse_out = ctx->row_lse;
-  CASCADE_TRY(launch_final_norm_mix(ctx, tree->T, hidden, hidden_f32, rms_gamma, eps, cfg_scale, 1.f / temperature, feat_out,
+  CASCADE_TRY(launch_final_norm_mix(ctx, tree->T, hidden, hidden_f32, add, rms_gamma, eps, cfg_scale, 1.f / temperature, feat_out,
                                     feat_norm_out, tok ? cand_parent_out : nullptr, tok ? cand_gparent_out : nullptr,
                                     s));
   if (ctx->shape.dtype == CASCADE_BF16) {
@@ -431,7 +431,8 @@ int cascade_lm_head_cfg(cascade_ctx* ctx, const cascade_tree* tree, const void* 
                         float* cand_parent_out, float* cand_gparent_out, void* stream) {
   if (ctx != nullptr) ctx->launches = 0;
   return lm_head_impl(ctx, tree, hidden, rms_gamma, eps, w_head, cfg_scale, temperature, tok, logits_out, feat_out,
-                      feat_norm_out, row_lse_out, cand_parent_out, cand_gparent_out, true, false, as_stream(stream));
+                      feat_norm_out, row_lse_out, cand_parent_out, cand_gparent_out, true, false, PendingAdd{},
+                      as_stream(stream));
 }
 
 // ---- (c) ------------------------------------------------------------------------------------------------
@@ -525,8 +526,9 @@ static int verify_step_impl(cascade_ctx* ctx, const cascade_tree* tree, const ca
   if (st->n_layers == 0 && st->hidden_in == nullptr) return CASCADE_ERR_INVALID_ARG;
   ctx->launches = 0;
   const void* hidden = st->hidden_in;
+  PendingAdd pending;
   if (st->n_layers > 0) {
-    CASCADE_TRY(run_layers(ctx, tree, st, s));
+    CASCADE_TRY(run_layers(ctx, tree, st, &pending, s));
     hidden = ctx->x;
   } else if (st->q != nullptr) {
     CASCADE_TRY(tree_attn_impl(ctx, tree, st->q, st->k_prefix, st->v_prefix, st->prefix_cap, st->prefix_len,
@@ -537,7 +539,7 @@ static int verify_step_impl(cascade_ctx* ctx, const cascade_tree* tree, const ca
   const bool bf16 = ctx->shape.dtype == CASCADE_BF16;
   CASCADE_TRY(lm_head_impl(ctx, tree, hidden, st->gamma_final, st->eps, st->w_head, st->cfg_scale, st->temperature,
                            st->tok, st->logits, feat, ctx->feat_norm, row_lse, ctx->cand_parent, ctx->cand_gparent, false,
-                           st->n_layers > 0, s));
+                           st->n_layers > 0, pending, s));
   // cosines, row log-sum-exp (bf16: folded from the head's partials), the rule and the path: one launch
   TailWork w;
   w.feat = feat;

@@ -206,8 +206,16 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
 
 // head.cu (norm + mix producers, fp32 head) / gemm_tc.cu (tcgen05 GEMM)
 // cand_parent / cand_gparent (may be null) are cleared here; the head fills the entries that exist.
-// hidden_f32: the hidden states are fp32 whatever the context's element type (the residual stream).
-int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidden_f32, const float* gamma, float eps,
+// Output matrices of a sliced projection that still have to be added to the residual stream.
+struct PendingAdd {
+  const float* slices = nullptr;  // [n][R*T][h]
+  int n = 0;
+  long long stride = 0;
+};
+// hidden_f32: the hidden states are fp32 whatever the context's element type (the residual stream); `add`
+// (fp32 hidden only) is added to them on the fly.
+int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidden_f32, const PendingAdd& add,
+                          const float* gamma, float eps,
                           float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
                           float* cand_parent, float* cand_gparent, cudaStream_t s);
 int launch_head_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* w_head, const int32_t* tok,
@@ -218,4 +226,6 @@ int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bflo
                      const int32_t* tok, float* logits, float* cand_parent, float* cand_gparent, cudaStream_t s);
 
 // layer.cu: the decoder layers of a verification step; leaves the residual stream in ctx->x.
-int run_layers(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, cudaStream_t s);
+// `pending`: the last MLP output, still to be added to ctx->x by whoever reads it next (empty if the
+// caller asked for the hidden states, in which case they are complete in ctx->x).
+int run_layers(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, PendingAdd* pending, cudaStream_t s);

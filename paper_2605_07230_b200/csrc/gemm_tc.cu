@@ -350,9 +350,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
         for (int c0 = 0; c0 < NB; c0 += 64) {
           const int n_cols = min(64, NB - c0);
           float v[64];
+          if (n_cols == 64) {
+            ptx::tmem_ld64(t_addr + c0, v);  // four loads in flight, one wait
+          } else {
 #pragma unroll
-          for (int sub = 0; sub < 4; ++sub)
-            if (16 * sub < n_cols) ptx::tmem_ld16(t_addr + c0 + 16 * sub, v + 16 * sub);
+            for (int sub = 0; sub < 4; ++sub)
+              if (16 * sub < n_cols) ptx::tmem_ld16(t_addr + c0 + 16 * sub, v + 16 * sub);
+          }
           if (contributor) {
             // partial of a split tile, [column][weight row]: coalesced over the lanes
             float* slot = p.sk_scratch + (((size_t)blockIdx.x * kHalves + half) * NB + c0) * kTileN + vl;
@@ -486,17 +490,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
 
 int64_t gemm_tc_scratch_floats(int sm_count) { return (int64_t)sm_count * 2 * 128 * kTileN; }
 
+// Accumulators (128 weight rows each) per work tile.  With more than 64 activation rows a stage holds
+// more activation bytes (high part and remainder, re-read from the L2 for every tile) than weight bytes,
+// and what an SM can take in per second, not HBM, bounds the weight stream: a 256-row tile feeds two
+// accumulators from one activation stage and halves that overhead.  Only the sliced mode does this (no
+// hand-off between CTAs, so TMEM need not hold a third accumulator set, and its matrices have many tiles).
+static int pick_halves(int NB, bool sliced) { return (sliced && NB > 64 && 4 * NB <= 512) ? 2 : 1; }
+
 int gemm_tc_pick_splits(int sm_count, int M, int N, int K, int max_splits) {
-  const int n_tiles = cascade_detail::ceil_div(N, kTileN) * cascade_detail::ceil_div(M, 128);
+  const OperandLayout lay = operand_layout(M, K);
+  const int halves = pick_halves(lay.NB, true);
+  const int n_tiles = cascade_detail::ceil_div(N, halves * kTileN) * lay.n_chunks;
   const int n_kb = cascade_detail::ceil_div(K, kSpan);
+  const long long kb_cost = halves * 16 + lay.NB / 4;  // KB an SM takes in per K block: weights + activation pair
   int best = 1;
   long long best_cost = -1;
   // a stage may carry two 64-wide K spans, and every slice needs at least one stage
   for (int s = 1; s <= max_splits && s <= cascade_detail::ceil_div(K, 2 * kSpan); ++s) {
-    // time ~ rounds x K blocks per item (8 cost units per K block of one round: 148 x 16 KB of weights),
-    // plus writing and re-reading one output matrix per slice at about the same rate
+    // time ~ rounds x K blocks per item, plus writing and re-reading one output matrix per slice at about
+    // the same rate
     const long long rounds = cascade_detail::ceil_div(n_tiles * s, sm_count);
-    const long long cost = rounds * cascade_detail::ceil_div(n_kb, s) * 8 + (long long)s * M * N / 37500;
+    const long long cost = rounds * cascade_detail::ceil_div(n_kb, s) * kb_cost + (long long)s * M * N / 6250;
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
       best = s;
@@ -529,9 +543,9 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   // A stage carries 32 KB of weights where three such stages fit (two K spans of a 128-row tile): the
   // round trip of the single producer / issue threads per stage limits the stream below that.  With
   // many activation rows the activation part of a stage is too large for that: one span per stage.
-  // (256-row tiles -- two accumulators per activation stage, half the activation traffic -- measured
-  // no faster on the stream and split the LM head of a 16384-token vocabulary over too few tiles.)
-  const int halves = 1;
+  // (With at most 64 activation rows, 256-row tiles measured no faster on the stream and split the LM
+  // head of a 16384-token vocabulary over too few tiles.)
+  const int halves = pick_halves(a.NB, epi.splits > 0);
   const int budget = 227 * 1024 - 20 * 1024 - 1024;  // static shared + alignment slack
   const int span_bytes = halves * kTileWBytes + 2 * a.NB * kSpan * 2;
   const int spans = (K % (2 * kSpan) == 0 && budget / (2 * span_bytes) >= 3) ? 2 : 1;
@@ -553,11 +567,13 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
       get_tmap_2d_bf16(ctx, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(halves * kTileN), kSpan);
   if (tw == nullptr) return CASCADE_ERR_CUDA;
   const int smem = a.stages * stage_bytes + 1024;
-  auto kern = spans == 2 ? k_gemm_tc<1, 2> : k_gemm_tc<1, 1>;
-  static int configured_smem[2] = {0, 0};
-  if (smem > configured_smem[spans - 1]) {
+  if (halves == 2 && spans == 2) return CASCADE_ERR_UNSUPPORTED_SHAPE;  // cannot happen: such stages do not fit
+  auto kern = halves == 2 ? k_gemm_tc<2, 1> : (spans == 2 ? k_gemm_tc<1, 2> : k_gemm_tc<1, 1>);
+  static int configured_smem[3] = {0, 0, 0};
+  const int kern_i = halves == 2 ? 2 : spans - 1;
+  if (smem > configured_smem[kern_i]) {
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    configured_smem[spans - 1] = smem;
+    configured_smem[kern_i] = smem;
   }
   long long grid = epi.splits > 0 ? (long long)n_tiles * epi.splits : a.units;
   if (grid > ctx->sm_count) grid = ctx->sm_count;

@@ -49,7 +49,9 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
                                                                  __nv_bfloat16* __restrict__ a_op,
                                                                  const OperandLayout lay, float* __restrict__ a_f32,
                                                                  float* __restrict__ cand_parent,
-                                                                 float* __restrict__ cand_gparent) {
+                                                                 float* __restrict__ cand_gparent,
+                                                                 const float* __restrict__ add, int n_add,
+                                                                 long long add_stride) {
   __shared__ float red[kNormThreads / 32];
   const int j = blockIdx.x, b = blockIdx.y;
   const size_t m = (size_t)b * T + j;
@@ -58,12 +60,27 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
   const int n8 = h / 8;
   float c[kNormChunks][8], u[kNormChunks][8];
   float ss_c = 0.f, ss_u = 0.f;
+  // 8 elements of the cond and the uncond row, plus whatever projection output has not been added to
+  // the residual stream yet
+  auto load_pair = [&](int i, float* vc, float* vu) {
+    load8(row_c + 8 * i, vc);
+    load8(row_u + 8 * i, vu);
+    for (int s2 = 0; s2 < n_add; ++s2) {
+      const float* a0 = add + (size_t)s2 * add_stride + 8 * (size_t)i;
+      float t[8];
+      load8(a0 + m * h, t);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) vc[e] += t[e];
+      load8(a0 + ((size_t)(B + b) * T + j) * h, t);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) vu[e] += t[e];
+    }
+  };
 #pragma unroll
   for (int k = 0; k < kNormChunks; ++k) {
     const int i = threadIdx.x + k * kNormThreads;
     if (i < n8) {
-      load8(row_c + 8 * i, c[k]);
-      load8(row_u + 8 * i, u[k]);
+      load_pair(i, c[k], u[k]);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         ss_c += c[k][e] * c[k][e];
@@ -73,8 +90,7 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
   }
   for (int i = threadIdx.x + kNormChunks * kNormThreads; i < n8; i += kNormThreads) {
     float tc[8], tu[8];
-    load8(row_c + 8 * i, tc);
-    load8(row_u + 8 * i, tu);
+    load_pair(i, tc, tu);
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
       ss_c += tc[e] * tc[e];
@@ -125,8 +141,7 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
   }
   for (int i = threadIdx.x + kNormChunks * kNormThreads; i < n8; i += kNormThreads) {
     float tc[8], tu[8];
-    load8(row_c + 8 * i, tc);
-    load8(row_u + 8 * i, tu);
+    load_pair(i, tc, tu);
     emit(i, tc, tu);
   }
   nn = block_sum(nn, red);
@@ -174,8 +189,8 @@ int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bflo
   return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a, sh.B * tree->T, e, K_GEMM_HEAD, s);
 }
 
-int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidden_f32, const float* gamma, float eps,
-                          float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
+int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidden_f32, const PendingAdd& add,
+                          const float* gamma, float eps, float cfg_scale, float inv_temperature, float* feat, float* feat_norm,
                           float* cand_parent, float* cand_gparent, cudaStream_t s) {
   const cascade_shape& sh = ctx->shape;
   dim3 grid(T, sh.B);
@@ -187,11 +202,12 @@ int launch_final_norm_mix(cascade_ctx* ctx, int T, const void* hidden, bool hidd
   if (bf16 && !hidden_f32)
     k_final_norm_mix<__nv_bfloat16><<<grid, kNormThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(hidden), sh.B, T,
                                                                   sh.h, gamma, eps, cfg_scale, inv_temperature, feat,
-                                                                  feat_norm, a_op, lay, a_f32, cand_parent, cand_gparent);
+                                                                  feat_norm, a_op, lay, a_f32, cand_parent, cand_gparent,
+                                                                  add.slices, add.n, add.stride);
   else
     k_final_norm_mix<float><<<grid, kNormThreads, 0, s>>>(static_cast<const float*>(hidden), sh.B, T, sh.h, gamma, eps,
                                                           cfg_scale, inv_temperature, feat, feat_norm, a_op, lay, a_f32,
-                                                          cand_parent, cand_gparent);
+                                                          cand_parent, cand_gparent, add.slices, add.n, add.stride);
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }

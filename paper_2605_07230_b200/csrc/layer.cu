@@ -130,8 +130,8 @@ __global__ void __launch_bounds__(kRowThreads) k_resid_norm(float* __restrict__ 
 
 // q, k, v = sum of the projection's slices; rotary embedding (half-split pairing: (x[i], x[i + D/2]) turned
 // by pos * base^(-2i/D)) on q and k at pos = prefix_len[r] + depth[j]; results in the attention's
-// element type.  grid (T, R): one position per CTA, so its D/2 (cos, sin) pairs are computed once into
-// shared memory.  D is a multiple of 8.
+// element type.  grid (T, R, z): one position per CTA, so its D/2 (cos, sin) pairs are computed once into
+// shared memory; the z CTAs of a row share its heads.  D is a multiple of 8.
 template <typename E>
 __global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restrict__ slices, int n_slices,
                                                             long long slice_stride, int T, int Hq, int Hkv, int D,
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restr
   };
   // rotated pairs of q and k, four pair indices per thread and step
   const int q4 = half / 4;
-  for (int t = threadIdx.x; t < (Hq + Hkv) * q4; t += kRowThreads) {
+  for (int t = blockIdx.z * kRowThreads + threadIdx.x; t < (Hq + Hkv) * q4; t += gridDim.z * kRowThreads) {
     const int head = t / q4, i = (t - head * q4) * 4;
     const int c0 = head * D + i;  // q heads first, then k heads: same column order as the projection
     const float4 x1 = col4(c0), x2 = col4(c0 + half);
@@ -185,7 +185,8 @@ __global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restr
       store4(k, o + half, y2);
     }
   }
-  for (int t = threadIdx.x; t < Hkv * D / 4; t += kRowThreads) store4(v, m * Hkv * D + 4 * t, col4((Hq + Hkv) * D + 4 * t));
+  for (int t = blockIdx.z * kRowThreads + threadIdx.x; t < Hkv * D / 4; t += gridDim.z * kRowThreads)
+    store4(v, m * Hkv * D + 4 * t, col4((Hq + Hkv) * D + 4 * t));
 }
 
 // act = silu(gate) * up from the slices of the fused gate/up projection ([.., 2*ffn]: gate then up).
@@ -273,7 +274,8 @@ int resid_norm(cascade_ctx* ctx, int T, const void* embed, const int32_t* tok, c
 }
 
 template <typename E>
-int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, cudaStream_t s) {
+int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, PendingAdd* pending,
+                 cudaStream_t s) {
   const cascade_shape& sh = ctx->shape;
   const int T = tree->T, R = 2 * sh.B, M = R * T;
   const int qkv_cols = (sh.Hq + 2 * sh.Hkv) * sh.D;
@@ -300,7 +302,8 @@ int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step*
     E* v_rot = st->v_tree_out ? (E*)st->v_tree_out + (size_t)li * M * sh.Hkv * sh.D : (E*)ctx->v_rot;
     {
       KernelScope ks(ctx, K_ROPE_SPLIT, s);
-      k_rope_split<E><<<dim3(T, R), kRowThreads, 0, s>>>(ctx->gemm_out, pr.n_slices, pr.slice_stride, T, sh.Hq, sh.Hkv,
+      const int z = cascade_detail::ceil_div((sh.Hq + sh.Hkv) * sh.D / 8, 2 * kRowThreads);  // ~2 pair groups per thread
+      k_rope_split<E><<<dim3(T, R, z < 1 ? 1 : z), kRowThreads, 0, s>>>(ctx->gemm_out, pr.n_slices, pr.slice_stride, T, sh.Hq, sh.Hkv,
                                                          sh.D, st->prefix_len, tree->d_depth, st->rope_base,
                                                          (E*)ctx->q_rot, k_rot, v_rot);
     }
@@ -330,17 +333,25 @@ int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step*
     CASCADE_CUDA_TRY(cudaGetLastError());
     CASCADE_TRY(project(ctx, L.w_down, sh.h, sh.ffn, M, false, K_GEMM_DOWN, &pr, s));
   }
-  // the last MLP output joins the residual stream; x is then the input of the final norm
+  // The last MLP output still has to join the residual stream.  The final norm adds it while it reads
+  // x; only a caller that wants the hidden states pays for a pass that writes them.
+  if (st->hidden_out == nullptr) {
+    pending->slices = ctx->gemm_out;
+    pending->n = pr.n_slices;
+    pending->stride = pr.slice_stride;
+    return CASCADE_OK;
+  }
+  *pending = PendingAdd{};
   return resid_norm<E>(ctx, T, nullptr, nullptr, &pr, nullptr, st->eps, st->hidden_out, K_RESID_ADD, s);
 }
 
 }  // namespace
 
-int run_layers(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, cudaStream_t s) {
+int run_layers(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* st, PendingAdd* pending, cudaStream_t s) {
   if (ctx->shape.ffn <= 0 || ctx->x == nullptr) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (st->layers == nullptr || st->embed == nullptr || st->prefix_len == nullptr) return CASCADE_ERR_INVALID_ARG;
   if (!(st->rope_base > 1.f) || !(st->softmax_scale > 0.f) || !(st->eps >= 0.f)) return CASCADE_ERR_INVALID_ARG;
   if (st->prefix_cap < 0 || st->prefix_cap > ctx->shape.P_max) return CASCADE_ERR_INVALID_ARG;
-  if (ctx->shape.dtype == CASCADE_BF16) return run_layers_t<__nv_bfloat16>(ctx, tree, st, s);
-  return run_layers_t<float>(ctx, tree, st, s);
+  if (ctx->shape.dtype == CASCADE_BF16) return run_layers_t<__nv_bfloat16>(ctx, tree, st, pending, s);
+  return run_layers_t<float>(ctx, tree, st, pending, s);
 }

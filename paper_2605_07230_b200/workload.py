@@ -139,8 +139,9 @@ class LayerWorkload:
 
     def __init__(self, w: synth.Workload, n_layers: int = 1, device="cuda:0", n_sets: int = 1,
                  keep_logits: bool = False, select_mode: int = cb.SELECT_LONGEST, flags: int = cb.USE_I | cb.USE_C,
-                 host: dict | None = None):
+                 host: dict | None = None, want_hidden: bool = True):
         self.w, self.device, self.n_layers = w, device, n_layers
+        self.want_hidden = want_hidden      # ask the step for the final hidden states (one more kernel)
         self.parent = w.parent()
         T = self.T = len(self.parent)
         self.ctx = cb.Context(cb.BF16 if w.dtype == "bf16" else cb.F32, w.B, T, max(w.prefix_len, 1), w.h, w.n_heads,
@@ -183,7 +184,8 @@ class LayerWorkload:
             q_relaxed=torch.zeros((B, T), device=dev), tvd_out=torch.zeros((B, T), device=dev),
             tvd_used=torch.zeros(B, device=dev), near_count=torch.zeros(B, dtype=torch.int32, device=dev),
             feat=torch.zeros((B, T, w.h), device=dev), scores=torch.zeros((B, max(self.tree.num_pairs, 1)), device=dev),
-            row_lse=torch.zeros((B, T), device=dev), hidden_out=torch.zeros((2 * B, T, w.h), device=dev),
+            row_lse=torch.zeros((B, T), device=dev),
+            hidden_out=torch.zeros((2 * B, T, w.h), device=dev) if self.want_hidden else None,
             k_tree_out=torch.zeros((self.n_layers, 2 * B, T, w.n_heads, w.head_dim), dtype=el, device=dev),
             v_tree_out=torch.zeros((self.n_layers, 2 * B, T, w.n_heads, w.head_dim), dtype=el, device=dev))
         if keep_logits or w.dtype != "bf16":
@@ -252,6 +254,7 @@ class DecodeLoop:
                                                                                      self.ctx, self.tree, self.params)
         w_cap = synth.Workload(**{**w.__dict__, "prefix_len": self.cap})
         wl.w = w_cap
+        wl.want_hidden = False                      # the loop has no use for the hidden states
         self.set = wl._make_set(host, True, select_mode)
         self.set.step.prefix_cap = self.cap
         self.u_bonus = torch.zeros(B, device=device)

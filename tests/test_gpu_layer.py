@@ -63,6 +63,23 @@ def test_step_through_layers(name, over, n_layers):
     wl.close()
 
 
+def test_step_without_hidden_output_matches():
+    """Without hidden_out the last MLP output is added inside the final norm (one kernel fewer): same
+    arithmetic in the same order, so logits, features and decisions are bit-identical."""
+    w = synth.workload("mini", B=2)
+    a = LayerWorkload(w, n_layers=2, keep_logits=True)
+    b = LayerWorkload(w, n_layers=2, keep_logits=True, want_hidden=False)
+    sa, sb = a.run(0), b.run(0)
+    torch.cuda.synchronize()
+    a.ctx.check()
+    b.ctx.check()
+    assert b.ctx.last_launch_count == a.ctx.last_launch_count - 1
+    for key in ("logits", "feat", "accept", "path_nodes", "path_len", "row_lse"):
+        assert torch.equal(sa.out[key], sb.out[key]), key
+    a.close()
+    b.close()
+
+
 def test_layers_need_stacked_projection_weights():
     w = synth.workload("mini", B=1)
     wl = LayerWorkload(w, n_layers=1)
