@@ -161,6 +161,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
       int slot = 0;
       uint32_t ph = 0;
+      const uint64_t pol_kv = ptx::l2_evict_first();  // the cache is read once per step
       for (int i = 0; i < n; ++i) {
         if (!ptx::mbar_wait(&empty[slot], ph ^ 1u, abort_flag, p.err)) break;
         const int tile = tile_begin + i;
@@ -169,8 +170,8 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys;
         uint8_t* dst = smem + ring_off + slot * kKVTileBytes;
         ptx::mbar_arrive_expect_tx(&full[slot], kKVTileBytes);
-        ptx::tma_load_4d(dst, m, 0, hk, key0, r, &full[slot]);
-        ptx::tma_load_4d(dst + kKVTileBytes / 2, m, 64, hk, key0, r, &full[slot]);
+        ptx::tma_load_4d_hint(dst, m, 0, hk, key0, r, &full[slot], pol_kv);
+        ptx::tma_load_4d_hint(dst + kKVTileBytes / 2, m, 64, hk, key0, r, &full[slot], pol_kv);
         if (++slot == slots) {
           slot = 0;
           ph ^= 1u;

@@ -171,6 +171,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
       int s = 0;
       uint32_t ph = 0;
       const int stages = p.stages, n_mchunks = p.n_mchunks, NB = p.NB;
+      const uint64_t pol_w = ptx::l2_evict_first(), pol_a = ptx::l2_evict_last();  // weights pass through once
       SegmentWalk walk(p);
       Segment sg;
       bool ok = true;
@@ -186,10 +187,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
           ptx::mbar_arrive_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
 #pragma unroll
           for (int q = 0; q < kSpans; ++q)
-            ptx::tma_load_2d(stage + q * kWSpanBytes, &tm_w, (kb * kSpans + q) * kSpan, n0, &full_bar[s]);
+            ptx::tma_load_2d_hint(stage + q * kWSpanBytes, &tm_w, (kb * kSpans + q) * kSpan, n0, &full_bar[s], pol_w);
           // the activations of these K blocks are contiguous in the staged layout: one bulk copy
-          ptx::bulk_load(stage + kWBytes, a_chunk + (size_t)kb * (kSpans * 2 * NB * kSpan), (uint32_t)(kSpans * a_span_bytes),
-                         &full_bar[s]);
+          ptx::bulk_load_hint(stage + kWBytes, a_chunk + (size_t)kb * (kSpans * 2 * NB * kSpan),
+                              (uint32_t)(kSpans * a_span_bytes), &full_bar[s], pol_a);
           if (++s == stages) {
             s = 0;
             ph ^= 1u;
