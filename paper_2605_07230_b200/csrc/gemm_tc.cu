@@ -132,7 +132,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ float st[kStCols * kStRow];
+  __shared__ __align__(16) float st[kStCols * kStRow];
   __shared__ int s_gather_n;
   __shared__ int4 s_gather[kGatherCap];  // {weight row in tile, parent column, grandparent column, idx}
 
@@ -320,6 +320,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
         if (n_tile * kTileN >= p.N) break;  // second half of the last work tile lies beyond N
         const int n = n_tile * kTileN + vl;
         const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (acc * kHalves + half) * (uint32_t)NB;
+        // plain result tiles that lie fully inside C with 16-byte aligned rows take the staged store
+        const bool wide_store = c_out != nullptr && !contributor && !e.accumulate && e.part == nullptr &&
+                                (e.ldc & 3) == 0 && (n_tile + 1) * kTileN <= p.N &&
+                                (reinterpret_cast<uintptr_t>(c_out) & 15u) == 0;
         int n_gather = 0;
         if (e.tok != nullptr && !contributor) {
           // which of the logits the acceptance rule reads (tok[idx] under its parent's and grandparent's
@@ -390,7 +394,28 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
               }
             }
           }
-          if (c_out != nullptr && n < p.N) {
+          if (wide_store) {
+            // Output rows are contiguous over the weight rows (n), a thread holds one n: staged through shared
+            // memory, a warp writes the 128 weight rows of an activation row with one 16-byte store per lane
+            // (a quarter of the store instructions of the direct path, each a full 512 bytes).
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              if (r * kStCols >= n_cols) break;
+              ptx::named_bar_sync(1, 128);  // the previous round has been read
+#pragma unroll
+              for (int i = 0; i < kStCols; ++i)
+                if (r * kStCols + i < n_cols) st[i * kTileN + vl] = v[r * kStCols + i];
+              ptx::named_bar_sync(1, 128);
+              const int row0 = m0 + c0 + r * kStCols;
+              float* dst = c_out + (size_t)row0 * e.ldc + n_tile * kTileN + 4 * lane;
+#pragma unroll
+              for (int k = 0; k < kStCols / 4; ++k) {
+                const int i = (warp - 2) + 4 * k;
+                if (r * kStCols + i < n_cols && row0 + i < p.M)
+                  *reinterpret_cast<float4*>(dst + (size_t)i * e.ldc) = *reinterpret_cast<const float4*>(st + i * kTileN + 4 * lane);
+              }
+            }
+          } else if (c_out != nullptr && n < p.N) {
             float* dst = c_out + (size_t)(m0 + c0) * e.ldc + n;
             const int rows = min(n_cols, p.M - (m0 + c0));  // rows of this group that exist
             if (e.accumulate) {
