@@ -57,6 +57,7 @@ struct GemmArgs {
   long long a_chunk_elems; // elements of one row chunk of A (all its K blocks)
   int stash;               // 1: TMEM has room for a third accumulator set (partials of split tiles)
   long long units;         // n_tiles * n_kb
+  int unit_q, unit_r;      // units = grid * unit_q + unit_r: CTA c starts at unit c * unit_q + min(c, unit_r)
   int n_tiles;
   int splits;              // 0: contiguous ranges with in-kernel hand-off; S >= 1: S K slices per tile
   long long slice_stride;  // floats between the C matrices of consecutive K slices
@@ -91,13 +92,16 @@ struct Segment {
 };
 // Contiguous mode (splits == 0): the flattened (tile, K block) list is cut into one range per CTA and
 // a segment is the part of a tile inside that range.  Sliced mode: work item w = (tile, K slice), taken
-// round-robin by the CTAs.
+// round-robin by the CTAs.  All of it in 32-bit arithmetic without a 64-bit division (the launcher checks
+// the ranges): this runs in single threads at the head of the kernel, before the first load can go out.
+// First unit of CTA c in contiguous mode.
+__device__ __forceinline__ int range_begin(const GemmArgs& p, int c) { return c * p.unit_q + min(c, p.unit_r); }
 struct SegmentWalk {
-  long long u, u_end;
+  int u, u_end;
   int n_kb, splits, w, n_items;
   __device__ SegmentWalk(const GemmArgs& p) : n_kb(p.n_kb), splits(p.splits) {
-    u = (long long)blockIdx.x * p.units / gridDim.x;
-    u_end = (long long)(blockIdx.x + 1) * p.units / gridDim.x;
+    u = range_begin(p, blockIdx.x);
+    u_end = range_begin(p, blockIdx.x + 1);
     w = blockIdx.x;
     n_items = p.n_tiles * p.splits;
   }
@@ -106,17 +110,17 @@ struct SegmentWalk {
       if (w >= n_items) return false;
       s.tile = w / splits;
       s.slice = w - s.tile * splits;
-      s.kb0 = (int)((long long)s.slice * n_kb / splits);
-      s.kb1 = (int)((long long)(s.slice + 1) * n_kb / splits);
+      s.kb0 = s.slice * n_kb / splits;
+      s.kb1 = (s.slice + 1) * n_kb / splits;
       w += gridDim.x;
       return true;
     }
     if (u >= u_end) return false;
     s.slice = 0;
-    s.tile = (int)(u / n_kb);
-    s.kb0 = (int)(u - (long long)s.tile * n_kb);
-    const long long left = u_end - u;
-    s.kb1 = left < (long long)(n_kb - s.kb0) ? s.kb0 + (int)left : n_kb;
+    s.tile = u / n_kb;
+    s.kb0 = u - s.tile * n_kb;
+    const int left = u_end - u;
+    s.kb1 = left < n_kb - s.kb0 ? s.kb0 + left : n_kb;
     u += s.kb1 - s.kb0;
     return true;
   }
@@ -209,6 +213,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
       SegmentWalk walk(p);
       Segment sg;
       bool ok = true;
+      // The first trip through the issue loop runs with every tensor-core instruction predicated off and
+      // waits for nothing: it only pulls the loop into the instruction cache (cold at every launch, the
+      // weights having streamed through the L2 since) while the first stage is still on its way.  The
+      // flag comes out of an asm statement so that the compiler keeps one copy of the loop.
+      uint32_t live;
+      asm volatile("mov.u32 %0, 0;" : "=r"(live));
       while (ok && walk.next(sg)) {
         const uint32_t acc = seg_i & 1u, aph = (seg_i >> 1) & 1u;
         ++seg_i;
@@ -217,11 +227,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
         const uint32_t d_tmem = tmem_base + acc * (uint32_t)(kHalves * p.NB);
         uint32_t accumulate = 0;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
-          if (!ptx::mbar_wait(&full_bar[s], ph, abort_flag, p.err)) {
-            ok = false;
-            break;
+          if (live != 0u) {
+            if (!ptx::mbar_wait(&full_bar[s], ph, abort_flag, p.err)) {
+              ok = false;
+              break;
+            }
+            ptx::tc_fence_after();
           }
-          ptx::tc_fence_after();
           const uint32_t w_addr = smem_base + (uint32_t)(s * stage_bytes);
 #pragma unroll
           for (int q = 0; q < kSpans; ++q) {
@@ -233,13 +245,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
 #pragma unroll
               for (int ks = 0; ks < kSpan / 16; ++ks) {
                 // advancing 16 K elements = 32 bytes = 2 descriptor units inside the swizzle span
-                ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + 2 * ks, idesc, (q | ks) == 0 ? accumulate : 1u);
-                ptx::umma_bf16(d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
+                ptx::umma_bf16_if(live, d, wd0 + 2 * ks, ad0 + 2 * ks, idesc, (q | ks) == 0 ? accumulate : 1u);
+                ptx::umma_bf16_if(live, d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
               }
             }
           }
+          ptx::umma_commit_if(live, &empty_bar[s]);  // stage reusable once these UMMAs have read it
+          if (live == 0u) {
+            asm volatile("mov.u32 %0, 1;" : "=r"(live));
+            --kb;  // now for real
+            continue;
+          }
           accumulate = 1u;
-          ptx::umma_commit(&empty_bar[s]);  // stage reusable once these UMMAs have read it
           if (++s == stages) {
             s = 0;
             ph ^= 1u;
@@ -274,8 +291,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
       const uint32_t stash_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(2 * kHalves * NB);
       if (owner_of_split) {
         // the CTAs after this one whose range starts inside this tile each hold one partial of it
-        const long long tile_end = (long long)(sg.tile + 1) * p.n_kb;
-        for (int c = blockIdx.x + 1; c < (int)gridDim.x && (long long)c * p.units / gridDim.x < tile_end; ++c) ++n_contrib;
+        const int tile_end = (sg.tile + 1) * p.n_kb;
+        for (int c = blockIdx.x + 1; c < (int)gridDim.x && range_begin(p, c) < tile_end; ++c) ++n_contrib;
         if (eid == 0) {
           for (int i = 1; i <= n_contrib && !*abort_flag; ++i) {
             const unsigned int* f = p.sk_flags + blockIdx.x + i;
@@ -603,6 +620,11 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   }
   long long grid = epi.splits > 0 ? (long long)n_tiles * epi.splits : a.units;
   if (grid > ctx->sm_count) grid = ctx->sm_count;
+  // the kernel's work assignment is 32-bit
+  if (a.units >= (1ll << 30) || (long long)a.n_kb * (epi.splits + 1) >= (1ll << 30) || (long long)n_tiles * (epi.splits + 1) >= (1ll << 30))
+    return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  a.unit_q = (int)(a.units / grid);
+  a.unit_r = (int)(a.units % grid);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(kThreads);
