@@ -58,7 +58,8 @@ constexpr int kKSlots = 2;     // K tiles in shared memory (a slot is free again
 constexpr int kVSlots = 3;     // V tiles in shared memory (free once O += P V has read it)
 constexpr int kPrefetch = 2;   // tiles requested into the L2 beyond what the shared-memory rings hold
 constexpr int kSmemBytes = kQBytes + kPBytes + (kKSlots + kVSlots) * kKVTileBytes + 1024;
-constexpr int kXRow = 133;  // row stride (floats) of the half-merge exchange buffer
+constexpr int kXRow = 132;  // row stride (floats) of the half-merge exchange buffer (16-byte aligned rows)
+constexpr int kORow = 132;  // row stride (floats) of the output staging buffer (16-byte aligned rows)
 
 struct AttnArgs {
   int T, Hq, Hkv, splits, n_rb, t_pad, prefix_cap;
@@ -139,7 +140,6 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
 
   // softmax state (warps 0-3)
-  float o_acc[kD];
   float m_run = -INFINITY, l_run = 0.f;
 
   if (warp == 4) {
@@ -344,52 +344,99 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       ptx::mbar_arrive(&p_full);
       l_run = l_run * alpha + rowsum;
     }
-#pragma unroll
-    for (int d = 0; d < kD; ++d) o_acc[d] = 0.f;
-    if (ok && n > 0) {
-      if (ptx::mbar_wait(&o_full, (n - 1) & 1u, abort_flag, p.err)) {
-        ptx::tc_fence_after();
-        ptx::tmem_ld64(o_addr, o_acc);
-        ptx::tmem_ld64(o_addr + 64, o_acc + 64);
-        ptx::tc_fence_before();
-      }
-    }
+    // The code from here to the end of the kernel runs once per CTA from a cold instruction cache, where
+    // every instruction line costs a fetch of its own: loops are rolled and the accumulator is taken from
+    // TMEM 16 columns at a time instead of as 128 registers.
+    bool have_o = false;
+    if (ok && n > 0) have_o = ptx::mbar_wait(&o_full, (n - 1) & 1u, abort_flag, p.err);
+    have_o = __all_sync(0xffffffffu, have_o);  // the TMEM loads below are warp-wide
+    ptx::tc_fence_after();
     // ---- merge the two key halves of each row (lanes r and r+64), then write ----
     // all UMMAs and TMA copies of this CTA have completed: the KV ring is free to reuse
-    float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);  // the K ring: 64 rows x 133 floats fit
+    float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);  // the K ring: 64 rows x kXRow floats fit
     ptx::named_bar_sync(1, 128);
     if (khalf == 1) {
       float* x = xbuf + row_in_block * kXRow;
+#pragma unroll 1
+      for (int c = 0; c < kD / 16; ++c) {
+        float v[16];
+        if (have_o) {
+          ptx::tmem_ld16(o_addr + 16 * c, v);
+        } else {
 #pragma unroll
-      for (int d = 0; d < kD; ++d) x[d] = o_acc[d];
+          for (int k = 0; k < 16; ++k) v[k] = 0.f;
+        }
+        float4* dst = reinterpret_cast<float4*>(x + 16 * c);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) dst[k] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+      }
       x[kD] = m_run;
       x[kD + 1] = l_run;
     }
     ptx::named_bar_sync(1, 128);
-    if (khalf == 0 && j < p.T) {
+    // Rows leave through shared memory: a thread holds a whole row here, and writing it directly would put
+    // 16 bytes per lane 512 bytes apart (measured: 5 us for 32 KB).  The Q / P area is idle by now.
+    float* obuf = reinterpret_cast<float*>(smem);  // [64 rows][kORow floats]
+    if (khalf == 0) {
       const float* x = xbuf + row_in_block * kXRow;
       const float m1 = x[kD], l1 = x[kD + 1];
       const float m = fmaxf(m_run, m1);
-      const float w0 = m_run == -INFINITY ? 0.f : ptx::ex2(m_run - m);
-      const float w1 = m1 == -INFINITY ? 0.f : ptx::ex2(m1 - m);
+      float w0 = m_run == -INFINITY ? 0.f : ptx::ex2(m_run - m);
+      float w1 = m1 == -INFINITY ? 0.f : ptx::ex2(m1 - m);
       const float l = l_run * w0 + l1 * w1;
-      if (p.splits == 1) {
+      if (p.splits == 1) {  // final values
         const float inv = 1.f / l;
-#pragma unroll
-        for (int c = 0; c < kD / 8; ++c) {
-          float v8[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) v8[k] = (o_acc[c * 8 + k] * w0 + x[c * 8 + k] * w1) * inv;
-          store8(p, r * p.T + j, head * kD + c * 8, p.Hq * kD, v8);
-        }
-      } else {
+        w0 *= inv;
+        w1 *= inv;
+      } else if (j < p.T) {
         const size_t unit = ((size_t)r * p.Hq + head) * p.splits + split;
-        float4* dst = reinterpret_cast<float4*>(p.part_o + (unit * p.t_pad + j) * kD);
-#pragma unroll
-        for (int c = 0; c < kD / 4; ++c)
-          dst[c] = make_float4(o_acc[4 * c] * w0 + x[4 * c] * w1, o_acc[4 * c + 1] * w0 + x[4 * c + 1] * w1,
-                               o_acc[4 * c + 2] * w0 + x[4 * c + 2] * w1, o_acc[4 * c + 3] * w0 + x[4 * c + 3] * w1);
         p.part_ml[unit * p.t_pad + j] = make_float2(m, l);
+      }
+      float* orow = obuf + row_in_block * kORow;
+#pragma unroll 1
+      for (int c = 0; c < kD / 16; ++c) {
+        float v[16];
+        if (have_o) {
+          ptx::tmem_ld16(o_addr + 16 * c, v);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 16; ++k) v[k] = 0.f;
+        }
+        if (j < p.T) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float4 xv = *reinterpret_cast<const float4*>(x + 16 * c + 4 * k);
+            *reinterpret_cast<float4*>(orow + 16 * c + 4 * k) =
+                make_float4(v[4 * k] * w0 + xv.x * w1, v[4 * k + 1] * w0 + xv.y * w1, v[4 * k + 2] * w0 + xv.z * w1,
+                            v[4 * k + 3] * w0 + xv.w * w1);
+          }
+        }
+      }
+    }
+    ptx::tc_fence_before();
+    ptx::named_bar_sync(1, 128);
+    if (p.splits == 1) {
+      // 16 pieces of 8 outputs per row; consecutive lanes take consecutive pieces (rolled: run-once code)
+#pragma unroll 1
+      for (int i = 0; i < 8; ++i) {
+        const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
+        const int jj = rb * kRowsPerBlock + row;
+        if (jj < p.T) {
+          const float4 a = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8);
+          const float4 b = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8 + 4);
+          const float v8[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+          store8(p, r * p.T + jj, head * kD + piece * 8, p.Hq * kD, v8);
+        }
+      }
+    } else {
+      const size_t unit = ((size_t)r * p.Hq + head) * p.splits + split;
+#pragma unroll 2
+      for (int i = 0; i < 16; ++i) {
+        const int idx = i * 128 + (int)threadIdx.x, row = idx >> 5, c4 = idx & 31;
+        const int jj = rb * kRowsPerBlock + row;
+        if (jj < p.T)
+          *reinterpret_cast<float4*>(p.part_o + (unit * p.t_pad + jj) * kD + 4 * c4) =
+              *reinterpret_cast<const float4*>(obuf + row * kORow + 4 * c4);
       }
     }
   }
@@ -414,54 +461,77 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (!s_last) return;
   __threadfence();
   if (threadIdx.x >= 128) return;
-  // out = sum_s w_s O_s / sum_s w_s l_s, w_s = 2^(m_s - max m), splits taken in index order
-  const int row = threadIdx.x & 63, j = rb * kRowsPerBlock + row, d0 = (threadIdx.x >> 6) * (kD / 2);
-  if (j >= p.T) return;
+  // out = sum_s w_s O_s / sum_s w_s l_s, w_s = 2^(m_s - max m), splits taken in index order.  The weights of a
+  // row go through shared memory, so that consecutive lanes can take consecutive 32-byte pieces of the
+  // partial outputs (a row per lane would read 16 bytes every 512).
   const size_t unit0 = ((size_t)r * p.Hq + head) * p.splits;
-  // two splits per round, every load of a round issued before the first use
-  float m = -INFINITY;
-  for (int s = 0; s < p.splits; ++s) m = fmaxf(m, __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + j]).x);
-  float acc[kD / 2];
-#pragma unroll
-  for (int d = 0; d < kD / 2; ++d) acc[d] = 0.f;
-  float l = 0.f;
-  for (int s0 = 0; s0 < p.splits; s0 += 2) {
-    const int s1 = min(s0 + 1, p.splits - 1);
-    const float2 ml0 = __ldcg(&p.part_ml[(unit0 + s0) * p.t_pad + j]);
-    const float2 ml1 = __ldcg(&p.part_ml[(unit0 + s1) * p.t_pad + j]);
-    const float4* src0 = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s0) * p.t_pad + j) * kD + d0);
-    const float4* src1 = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s1) * p.t_pad + j) * kD + d0);
-    float4 t0[kD / 8], t1[kD / 8];
-#pragma unroll
-    for (int c = 0; c < kD / 8; ++c) t0[c] = __ldcg(src0 + c);
-#pragma unroll
-    for (int c = 0; c < kD / 8; ++c) t1[c] = __ldcg(src1 + c);
-    const float w0 = ml0.x == -INFINITY ? 0.f : ptx::ex2(ml0.x - m);
-    const float w1 = (s1 == s0 || ml1.x == -INFINITY) ? 0.f : ptx::ex2(ml1.x - m);
-    l += w0 * ml0.y;
-    l += w1 * ml1.y;
-#pragma unroll
-    for (int c = 0; c < kD / 8; ++c) {
-      acc[4 * c] += w0 * t0[c].x;
-      acc[4 * c + 1] += w0 * t0[c].y;
-      acc[4 * c + 2] += w0 * t0[c].z;
-      acc[4 * c + 3] += w0 * t0[c].w;
-    }
-#pragma unroll
-    for (int c = 0; c < kD / 8; ++c) {
-      acc[4 * c] += w1 * t1[c].x;
-      acc[4 * c + 1] += w1 * t1[c].y;
-      acc[4 * c + 2] += w1 * t1[c].z;
-      acc[4 * c + 3] += w1 * t1[c].w;
+  float* s_w = reinterpret_cast<float*>(smem);  // [splits][64] weights, then [64] 1 / sum
+  float* s_inv = s_w + p.splits * kRowsPerBlock;
+  if (threadIdx.x < kRowsPerBlock) {
+    const int row = threadIdx.x, jj = rb * kRowsPerBlock + row;
+    if (jj < p.T) {
+      float m = -INFINITY;
+      for (int s = 0; s < p.splits; ++s) m = fmaxf(m, __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + jj]).x);
+      float l = 0.f;
+      for (int s = 0; s < p.splits; ++s) {
+        const float2 ml = __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + jj]);
+        const float w = ml.x == -INFINITY ? 0.f : ptx::ex2(ml.x - m);
+        s_w[s * kRowsPerBlock + row] = w;
+        l += w * ml.y;
+      }
+      s_inv[row] = 1.f / l;
     }
   }
-  const float inv = 1.f / l;
+  ptx::named_bar_sync(1, 128);
+  float acc[8][8];
 #pragma unroll
-  for (int c = 0; c < kD / 16; ++c) {
-    float v8[8];
+  for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int k = 0; k < 8; ++k) v8[k] = acc[8 * c + k] * inv;
-    store8(p, r * p.T + j, head * kD + d0 + c * 8, p.Hq * kD, v8);
+    for (int k = 0; k < 8; ++k) acc[i][k] = 0.f;
+  for (int s = 0; s < p.splits; ++s) {
+    float4 t[8][2];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {  // every load of this split issued before the first use
+      const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
+      const int jj = min(rb * kRowsPerBlock + row, p.T - 1);
+      const float4* src = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s) * p.t_pad + jj) * kD + piece * 8);
+      t[i][0] = __ldcg(src);
+      t[i][1] = __ldcg(src + 1);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float w = s_w[s * kRowsPerBlock + ((i * 128 + (int)threadIdx.x) >> 4)];
+      acc[i][0] += w * t[i][0].x;
+      acc[i][1] += w * t[i][0].y;
+      acc[i][2] += w * t[i][0].z;
+      acc[i][3] += w * t[i][0].w;
+      acc[i][4] += w * t[i][1].x;
+      acc[i][5] += w * t[i][1].y;
+      acc[i][6] += w * t[i][1].z;
+      acc[i][7] += w * t[i][1].w;
+    }
+  }
+  // The sums go back to shared memory and leave through a short rolled loop: this code runs once per CTA
+  // from a cold instruction cache, and every instruction line of an unrolled version costs a fetch.
+  float* obuf = s_inv + kRowsPerBlock;  // [64 rows][kORow floats]
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
+    float4* dst = reinterpret_cast<float4*>(obuf + row * kORow + piece * 8);
+    dst[0] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    dst[1] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+  }
+  __syncwarp();  // a thread reads back only what it wrote
+#pragma unroll 1
+  for (int i = 0; i < 8; ++i) {
+    const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
+    const int jj = rb * kRowsPerBlock + row;
+    if (jj >= p.T) continue;
+    const float inv = s_inv[row];
+    const float4 a = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8);
+    const float4 b = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8 + 4);
+    const float v8[8] = {a.x * inv, a.y * inv, a.z * inv, a.w * inv, b.x * inv, b.y * inv, b.z * inv, b.w * inv};
+    store8(p, r * p.T + jj, head * kD + piece * 8, p.Hq * kD, v8);
   }
 }
 
