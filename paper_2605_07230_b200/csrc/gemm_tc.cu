@@ -331,7 +331,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
       }
       if (!ptx::mbar_wait(&tmem_full[acc], aph, abort_flag, p.err)) break;
       ptx::tc_fence_after();
-#pragma unroll
+#pragma unroll 1  // run-once code: the second half re-uses the instruction lines of the first
       for (int half = 0; half < kHalves; ++half) {
         const int n_tile = macro * kHalves + half;
         if (n_tile * kTileN >= p.N) break;  // second half of the last work tile lies beyond N
