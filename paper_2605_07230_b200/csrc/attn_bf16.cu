@@ -91,6 +91,13 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t q_addr = smem_base, p_addr = smem_base + kQBytes, k_ring = p_addr + kPBytes,
                  v_ring = k_ring + kKSlots * kKVTileBytes;
 
+  if (threadIdx.x == 128) {  // the TMA warp's first loads should not wait for their descriptors
+    ptx::prefetch_tmap(&tm_q);
+    ptx::prefetch_tmap(&tm_kp);
+    ptx::prefetch_tmap(&tm_vp);
+    ptx::prefetch_tmap(&tm_kt);
+    ptx::prefetch_tmap(&tm_vt);
+  }
   const int split = blockIdx.x, head = blockIdx.y / p.n_rb, rb = blockIdx.y % p.n_rb, r = blockIdx.z;
   const int hk = head / (p.Hq / p.Hkv);
   const int P = p.prefix_len[r];
