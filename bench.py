@@ -19,6 +19,7 @@ prompts, so there is nothing to shard or reduce); the time is the max over ranks
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import sys
@@ -26,6 +27,17 @@ import threading
 import time
 
 import numpy as np
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
+# (step_kernels_layer_*_full.txt: default step, one launch of each kernel), and the first 16 hex digits of
+# the SHA-256 of the kernel source they were taken on.  A kernel whose source has changed since reports
+# "traffic": null.
+NCU_TRAFFIC = {
+    "janus": {"gemm_qkv": 107809280, "tree_attn": 15641344, "gemm_o": 35745024, "gemm_gate_up": 192148224,
+              "gemm_down": 100870912, "gemm_head": 139382016},
+    "lumina": {},
+}
+NCU_TRAFFIC_SOURCES = {"gemm_tc.cu": "a17cadb3f98c3964", "attn_bf16.cu": "9f1b130524f96247"}
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
@@ -325,11 +337,23 @@ def main():
     per_kernel = {k: {"us": 1e3 * v[0] / v[1], "launches_per_step": v[1] / kt_steps} for k, v in timing.items()}
     step_us_kernels = sum(1e3 * v[0] for v in timing.values()) / kt_steps
     dom = max((k for k in timing if k in alg_b), key=lambda k: timing[k][0])
+    def traffic(k):
+        # dram bytes per launch from the ncu capture summarised under profiles/: only for the step they were
+        # taken on (layer mode) and only while the kernel's source is what it was then
+        if args.mode != "layer" or k not in NCU_TRAFFIC.get(args.workload, {}):
+            return None
+        src = "attn_bf16.cu" if k == "tree_attn" else "gemm_tc.cu"
+        path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2605_07230_b200", "csrc", src)
+        with open(path, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != NCU_TRAFFIC_SOURCES[src]:
+                return None
+        return NCU_TRAFFIC[args.workload][k]
+
     def roof(k):
         us = per_kernel[k]["us"]
         ach = alg_b[k] / (us * 1e-6) / 1e9
         d = {"kernel": k, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-             "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"], "us_per_launch": us,
+             "frac": ach / peaks["hbm_gbs"], "traffic": traffic(k), "peak_source": peaks["source"], "us_per_launch": us,
              "algorithmic_bytes": alg_b[k]}
         if k in alg_f:
             d["tensor_tflops"] = alg_f[k] / (us * 1e-6) / 1e12
