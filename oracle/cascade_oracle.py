@@ -16,7 +16,8 @@ Where the paper is silent or inconsistent the reading taken is stated at the fun
 Parity pins (tests/test_oracle_*.py): every function below is pinned to something outside itself:
 textbook causal / decode attention, CFG end points and linearity, closed-form cosine cases, reduction
 to Algorithm 1 with the relaxation off, an independently written sequential walk of Algorithm 2,
-brute-force path enumeration, threshold monotonicity with an unbounded budget, hand-computed trees.
+brute-force path enumeration, threshold monotonicity with an unbounded budget, hand-computed trees,
+the library's top-k and a brute-force nucleus for the truncation of the target distribution.
 `decoder_layer` is pinned only through special cases (zero weights -> identity; the rotary map is
 checked against complex multiplication); the architecture itself comes from the workload definition,
 not from the paper.
@@ -375,6 +376,40 @@ def bonus_token(logits_row, rejected_tokens, u):
     c = np.cumsum(g)
     v = int(np.searchsorted(c, float(u) * total, side="right"))
     return min(v, len(g) - 1), total
+
+
+def filter_logits(logits, top_k, top_p):
+    """Top-k / nucleus truncation of the target distribution before verification (the sampling settings
+    of the paper's experiments, Appendix D.1: temperature 1, top-p 1.0, top-k 2000; the paper gives the
+    numbers only, the truncations are the usual ones, stated here so that ties are decided).  Per row:
+      top-k (0 < top_k < V): keep every token whose logit is >= the top_k-th largest logit of the row
+        (tokens tied with it stay together, so more than top_k can remain);
+      top-p (top_p < 1), on the distribution renormalised over what top-k kept: keep a token iff the
+        probability of the tokens with a strictly larger logit is < top_p (the smallest set of most
+        likely tokens whose mass reaches top_p; ties stay together).
+    Dropped tokens get logit -inf, i.e. probability zero after the softmax.  Returns (filtered, kept)."""
+    logits = np.asarray(logits, np.float64)
+    V = logits.shape[-1]
+    flat = logits.reshape(-1, V)
+    out = flat.copy()
+    kept = np.ones(flat.shape, bool)
+    for i, row in enumerate(flat):
+        keep = np.ones(V, bool)
+        if 0 < top_k < V:
+            kth = np.sort(row)[V - top_k]
+            keep &= row >= kth
+        if top_p < 1.0:
+            p = softmax(np.where(keep, row, -np.inf))
+            order = np.argsort(-row, kind="stable")
+            sorted_l, sorted_p = row[order], p[order]
+            before = np.cumsum(sorted_p) - sorted_p              # mass ahead of each position
+            first_of_value = np.searchsorted(-sorted_l, -sorted_l, side="left")  # ties share the first position
+            larger = np.empty(V)
+            larger[order] = before[first_of_value]
+            keep &= larger < top_p
+        kept[i] = keep
+        out[i, ~keep] = -np.inf
+    return out.reshape(logits.shape), kept.reshape(logits.shape)
 
 
 def append_path_kv(k_cache, v_cache, prefix_len, k_tree, v_tree, path, B):
