@@ -323,6 +323,25 @@ int cascade_kv_append(cascade_ctx* ctx, const cascade_tree* tree, int32_t n_laye
                       const void* k_tree, const void* v_tree, const int32_t* path_nodes, const int32_t* path_len,
                       int32_t prefix_cap, int32_t* prefix_len, void* stream);
 
+/* ---- truncation of the target distribution ------------------------------------------------------- */
+/* Top-k / nucleus truncation of target logits, in place (the sampling settings of the paper's experiments,
+ * Appendix D.1: temperature 1, top-p 1.0, top-k 2000; the paper states the numbers, the truncations are
+ * the usual ones).  Per row of V logits:
+ *   top_k (0 < top_k < V; 0 or >= V: off): keep the tokens whose logit is >= the top_k-th largest logit of the
+ *     row -- tokens tied with it stay together, so more than top_k can remain;
+ *   top_p (< 1; 1: off), on the distribution renormalised over what top-k kept: keep a token iff the
+ *     probability of the tokens with a strictly larger logit is < top_p (ties stay together).
+ * A dropped token's logit becomes -inf: cascade_relaxed_accept (with these logits), cascade_bonus_token and
+ * any softmax over the row then give it probability zero and renormalise the rest.
+ *   logits [n_rows, V] float, DEVICE, read and written (V from the context's shape; rows are independent,
+ *          e.g. the [B,T,V] logits of cascade_lm_head_cfg with n_rows = B*T);
+ *   kept_count [n_rows] int32 DEVICE or NULL: how many tokens of each row remain.
+ * Both thresholds are exact (a radix descent over the logits' bit patterns; the nucleus sums probabilities
+ * in 40-bit fixed point, so the result does not depend on the order of the additions).
+ * Errors: CASCADE_ERR_INVALID_ARG (null pointers, n_rows < 1, top_k < 0, top_p outside (0, 1]). */
+int cascade_filter_logits(cascade_ctx* ctx, float* logits, int32_t n_rows, int32_t top_k, float top_p,
+                          int32_t* kept_count, void* stream);
+
 /* ---- acceptance without any device allocation --------------------------------------------------- */
 /* The paper has no counterpart to this entry point; it exists for deployment.  Some callers of this
  * library may not allocate device memory at all: a plug-in running inside a serving process that

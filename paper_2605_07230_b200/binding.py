@@ -29,6 +29,7 @@ EXPORTS = [
     "cascade_tree_num_pairs", "cascade_tree_pairs", "cascade_tree_attn", "cascade_lm_head_cfg",
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
     "cascade_verify_step_host", "cascade_accept_static", "cascade_bonus_token", "cascade_kv_append",
+    "cascade_filter_logits",
 ]
 
 
@@ -102,6 +103,7 @@ def lib() -> C.CDLL:
                                             C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.cascade_bonus_token.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.cascade_kv_append.argtypes = [vp, vp, C.c_int32, C.POINTER(Layer), vp, vp, vp, vp, C.c_int32, vp, vp]
+        L.cascade_filter_logits.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_float, vp, vp]
         _lib = L
     return _lib
 
@@ -295,6 +297,12 @@ def cascade_accept_static(B, parent, feat, feat_dim, feat_norm, row_lse, cand_pa
                                        _ptr(uniforms), C.byref(params), select_mode, _ptr(accept), _ptr(q_relaxed),
                                        _ptr(tvd_out), _ptr(near_count), _ptr(path_nodes), _ptr(path_len),
                                        _ptr(tvd_used), _stream()))
+
+
+def cascade_filter_logits(ctx, logits, top_k, top_p, kept_count=None):
+    n_rows = logits.numel() // logits.shape[-1]
+    _check(lib().cascade_filter_logits(ctx.handle, _ptr(logits), n_rows, int(top_k), float(top_p), _ptr(kept_count),
+                                       _stream()))
 
 
 def cascade_bonus_token(ctx, tree, logits, tok, path_nodes, path_len, u_bonus, token_out, mass_out=None):

@@ -147,7 +147,7 @@ const char* cascade_kernel_name(int32_t id) {
   static const char* names[] = {"tree_attn", "tree_attn_f32", "final_norm_mix", "gemm_head",
                                 "head_f32", "row_stats", "row_lse", "similarity", "accept", "tail", "select_path",
                                 "embed_norm", "gemm_qkv", "rope_split", "gemm_o", "resid_norm", "gemm_gate_up",
-                                "swiglu", "gemm_down", "gemm_f32", "resid_add", "kv_append", "bonus_token"};
+                                "swiglu", "gemm_down", "gemm_f32", "resid_add", "kv_append", "bonus_token", "filter_logits"};
   static_assert(sizeof(names) / sizeof(names[0]) == K_KERNEL_ID_END, "one name per kernel id");
   if (id < 0 || id >= K_KERNEL_ID_END) return nullptr;
   return names[id];

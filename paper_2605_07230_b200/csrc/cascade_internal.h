@@ -35,7 +35,7 @@ enum KernelId : int {
   K_TREE_ATTN = 0, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_GEMM_HEAD, K_HEAD_F32, K_ROW_STATS,
   K_ROW_LSE, K_SIMILARITY, K_ACCEPT, K_TAIL, K_SELECT_PATH, K_EMBED_NORM, K_GEMM_QKV, K_ROPE_SPLIT, K_GEMM_O,
   K_RESID_NORM, K_GEMM_GATE_UP, K_SWIGLU, K_GEMM_DOWN, K_GEMM_F32, K_RESID_ADD, K_KV_APPEND, K_BONUS_TOKEN,
-  K_KERNEL_ID_END
+  K_FILTER_LOGITS, K_KERNEL_ID_END
 };
 static_assert(K_KERNEL_ID_END <= CASCADE_KERNEL_COUNT, "timing table too small");
 
