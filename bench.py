@@ -194,6 +194,8 @@ def main():
                     help="layer: the step runs through one decoder layer; pieces: the four named pieces alone")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every step from Python instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--top-k", type=int, default=2000,
+                    help="also time cascade_filter_logits (top-k truncation of the target logits, outside the step); 0 = skip")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets (0 = enough to exceed the L2 per step)")
     args = ap.parse_args()
 
@@ -285,6 +287,30 @@ def main():
         timing = wl.ctx.timing_read()
         wl.ctx.timing_enable(False)
         clocks = sampler.stop()
+
+        # top-k truncation of the target distribution (the paper's sampling setting; not part of the timed step)
+        filter_info = None
+        if args.top_k > 0:
+            gen = torch.Generator(device=dev).manual_seed(w.seed)
+            centres = torch.randn(256, generator=gen, device=dev)
+            rows_f = w.B * T
+            base = centres[torch.arange(w.V, device=dev) % 256][None, :] * (8.0 / 3.0) + \
+                0.3 * torch.randn((rows_f, w.V), generator=gen, device=dev)
+            copies = [base.clone() for _ in range(22)]
+            cb.cascade_filter_logits(wl.ctx, copies[0], args.top_k, 1.0)
+            cb.cascade_filter_logits(wl.ctx, copies[1], args.top_k, 1.0)
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record(stream)
+            for c in copies[2:]:
+                cb.cascade_filter_logits(wl.ctx, c, args.top_k, 1.0)
+            f1.record(stream)
+            stream.synchronize()
+            wl.ctx.check()
+            filter_info = {"top_k": args.top_k, "top_p": 1.0, "rows": rows_f, "V": w.V,
+                           "us_per_call": 1e3 * f0.elapsed_time(f1) / 20, "logits_bytes": rows_f * w.V * 4,
+                           "kept_per_row": int((~torch.isinf(copies[2][0])).sum()), "bound": "latency",
+                           "note": "stand-alone call on [B*T, V] fp32 logits resident in the L2"}
+            del copies, base
 
         # end to end through the host-buffer entry: pinned host inputs in, results out, every step
         s0 = wl.sets[0]
@@ -381,6 +407,7 @@ def main():
         "accepted_tokens_per_step": alpha_sum / (e2e_steps * w.B),
         "e2e": {"value": world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * done,
+        "filter_logits": filter_info,
         "launches_per_step": launches_per_step,
         "kernels_us": {k: round(v["us"], 3) for k, v in sorted(per_kernel.items())},
         "kernel_time_per_step_us": step_us_kernels, "dominant_kernel": dom,
