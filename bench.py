@@ -30,14 +30,13 @@ import numpy as np
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
 # (step_kernels_layer_*_full.txt: default step, one launch of each kernel), and the first 16 hex digits of
-# the SHA-256 of the kernel source they were taken on.  A kernel whose source has changed since reports
+# the SHA-256 of the kernel sources (the .cu file, ptx.cuh, operand.cuh) they were taken on.  A kernel whose source has changed since reports
 # "traffic": null.
 NCU_TRAFFIC = {
-    "janus": {"gemm_qkv": 107809280, "tree_attn": 15641344, "gemm_o": 35745024, "gemm_gate_up": 192148224,
-              "gemm_down": 100870912, "gemm_head": 139382016},
-    "lumina": {},
+    "janus": {"gemm_qkv": 107990784, "tree_attn": 15641600, "gemm_o": 35746304, "gemm_gate_up": 190910464, "gemm_down": 100720384, "gemm_head": 139390720},
+    "lumina": {"gemm_qkv": 108056064, "tree_attn": 87570688, "gemm_o": 35733760, "gemm_gate_up": 190966016, "gemm_down": 100879616, "gemm_head": 544727040},
 }
-NCU_TRAFFIC_SOURCES = {"gemm_tc.cu": "a17cadb3f98c3964", "attn_bf16.cu": "9f1b130524f96247"}
+NCU_TRAFFIC_SOURCES = {"gemm_tc.cu": "4c12780f9a7d5bd0", "attn_bf16.cu": "028d7c3df0005695"}
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
@@ -369,10 +368,13 @@ def main():
         if args.mode != "layer" or k not in NCU_TRAFFIC.get(args.workload, {}):
             return None
         src = "attn_bf16.cu" if k == "tree_attn" else "gemm_tc.cu"
-        path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2605_07230_b200", "csrc", src)
-        with open(path, "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest()[:16] != NCU_TRAFFIC_SOURCES[src]:
-                return None
+        csrc = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2605_07230_b200", "csrc")
+        digest = hashlib.sha256()
+        for name in (src, "ptx.cuh", "operand.cuh"):   # the kernel and the headers its device code comes from
+            with open(os.path.join(csrc, name), "rb") as f:
+                digest.update(f.read())
+        if digest.hexdigest()[:16] != NCU_TRAFFIC_SOURCES[src]:
+            return None
         return NCU_TRAFFIC[args.workload][k]
 
     def roof(k):
