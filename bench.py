@@ -182,6 +182,74 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def run_loop(args, dev, peaks, rank, world):
+    """The last workload of the set: a speculative decode loop through `--layers` decoder layers at the
+    Janus-shaped widths, prompt cache 64 rows growing by the accepted tokens.  A step = cascade_verify_step
+    (all layers, head, acceptance, path) + cascade_bonus_token + cascade_kv_append; the stand-in drafter and
+    the read-back of path and token run on the host between steps and are outside the device time.
+    Every layer has its own weights and caches on the device (12 GB at 30 layers); the values of the
+    layers' weights are those of one seeded layer (see DecodeLoop)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2605_07230_b200 import synth
+    from paper_2605_07230_b200.workload import DecodeLoop
+
+    K, W = min(args.steps, 78), 4                      # 64 + 82 * 7 = 638 cache rows: the workload's 64 -> 64 + 576
+    w = synth.workload("janus", prefix_len=64)
+    loop = DecodeLoop(w, n_layers=args.layers, max_steps=K + W, device=dev, seed=5, tile_layers=True)
+    for _ in range(W):
+        loop.step()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(int(dev.split(":")[1]))
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    accepted = 0
+    t0 = time.perf_counter()
+    for i in range(K):
+        drafted = loop.draft()
+        ev[i][0].record()
+        out = loop.step(drafted, events_after=ev[i][1])
+        accepted += int(out["path_len"].sum())
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    clocks = sampler.stop()
+    dev_ms = sum(a.elapsed_time(b) for a, b in ev)
+    launches = loop.launches_last_step * K
+    if world > 1:
+        t = torch.tensor([dev_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dev_ms = float(t.item())
+    loop.close()
+    if rank != 0:
+        return
+    hd = w.n_heads * w.head_dim
+    layer_bytes = (4 * hd * w.h + 3 * w.ffn * w.h) * 2
+    step_bytes = args.layers * layer_bytes + w.V * w.h * 2
+    value = world * K / (dev_ms * 1e-3)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": "loop", "layers": args.layers, "B": w.B, "tree_rows": loop.T, "prefix_len": "64 -> %d" % int(loop.prefix_len_host[0]),
+                   "V": w.V, "h": w.h, "ffn": w.ffn, "heads": w.n_heads, "head_dim": w.head_dim,
+                   "step": "verify step through all layers + bonus token + cache append; drafter and read-back on the host, outside the device time",
+                   "l2": "each layer streams its own 405 MB of weights (> 126 MB L2)", "cuda_graph": False,
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "accepted_tokens_per_step": accepted / (K * w.B), "tokens_per_step_with_bonus": accepted / (K * w.B) + 1,
+        "tokens_per_s": value * (accepted / (K * w.B) + 1),
+        "e2e": {"value": world * K / wall, "unit": UNIT, "h2d_bytes_per_step": 3 * w.B * loop.T * 4 + 4 * w.B,
+                "d2h_bytes_per_step": w.B * (loop.tree.depth + 1) * 4 + 8 * w.B,
+                "note": "wall clock per step including the host drafter, the copies of its output and the read-back of path and token"},
+        "gpu_launches": launches,
+        "step_roofline": {"algorithmic_bytes": step_bytes, "floor_us": step_bytes / peaks["hbm_gbs"] / 1e3,
+                          "frac_of_hbm_floor": step_bytes / peaks["hbm_gbs"] / 1e3 / (1e3 * dev_ms / K)},
+        "roofline": None, "cpu_baseline": None, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -189,8 +257,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default="janus")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--mode", default="layer", choices=["layer", "pieces"],
-                    help="layer: the step runs through one decoder layer; pieces: the four named pieces alone")
+    ap.add_argument("--mode", default="layer", choices=["layer", "pieces", "loop"],
+                    help="layer: the step runs through one decoder layer; pieces: the four named pieces alone; "
+                         "loop: a 30-layer speculative decode loop (verify, bonus token, cache append each step)")
+    ap.add_argument("--layers", type=int, default=30, help="decoder layers in --mode loop")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every step from Python instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--top-k", type=int, default=2000,
@@ -217,6 +287,11 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     dev = f"cuda:{local}"
     peaks = load_peaks()
+    if args.mode == "loop":
+        run_loop(args, dev, peaks, rank, world)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # enough rotating copies of the inputs that a step never finds its operands in the 126 MB L2
     parent = w.parent()

@@ -226,7 +226,9 @@ class DecodeLoop:
     argument marshalling only."""
 
     def __init__(self, w: synth.Workload, n_layers: int, max_steps: int, device="cuda:0", seed: int = 0,
-                 select_mode: int = cb.SELECT_LONGEST):
+                 select_mode: int = cb.SELECT_LONGEST, tile_layers: bool = False):
+        # tile_layers: every layer gets the values of one seeded layer (its own copy on the device, its own
+        # caches): for timing at full depth without generating 30 layers of weights on the host
         self.w, self.n_layers, self.device = w, n_layers, device
         self.parent = w.parent()
         T = self.T = len(self.parent)
@@ -238,7 +240,13 @@ class DecodeLoop:
         self.tree = cb.Tree(self.ctx, self.parent)
         self.params = cb.Params(w.tau_pos, w.tau_seq, w.tvd_budget, cb.USE_I | cb.USE_C)
         rng = np.random.default_rng(w.seed)
-        host = synth.layer_step_inputs(w, rng, self.parent, n_layers)
+        if tile_layers:
+            host = synth.layer_step_inputs(w, rng, self.parent, 1)
+            host["layers"] = host["layers"] * n_layers
+            host["k_prefix"] = [host["k_prefix"][0]] * n_layers
+            host["v_prefix"] = [host["v_prefix"][0]] * n_layers
+        else:
+            host = synth.layer_step_inputs(w, rng, self.parent, n_layers)
         # caches with room for the whole run; the first prefix_len rows hold the seeded prompt cache
         for li in range(n_layers):
             for name in ("k_prefix", "v_prefix"):
@@ -270,7 +278,7 @@ class DecodeLoop:
         ub = self.rng.random(w.B, dtype=np.float32)
         return tok, p, u, ub
 
-    def step(self, drafted=None):
+    def step(self, drafted=None, events_after=None):
         tok, p, u, ub = drafted if drafted is not None else self.draft()
         d, o = self.set.dev, self.set.out
         d["tok"].copy_(torch.from_numpy(tok))
@@ -278,10 +286,15 @@ class DecodeLoop:
         d["uniforms"].copy_(torch.from_numpy(u))
         self.u_bonus.copy_(torch.from_numpy(ub))
         cb.cascade_verify_step(self.ctx, self.tree, self.set.step)
+        n_launch = self.ctx.last_launch_count
         cb.cascade_bonus_token(self.ctx, self.tree, o["logits"], d["tok"], o["path_nodes"], o["path_len"], self.u_bonus,
                                self.bonus, self.mass)
+        n_launch += self.ctx.last_launch_count
         cb.cascade_kv_append(self.ctx, self.tree, self.set.step, o["k_tree_out"], o["v_tree_out"], o["path_nodes"],
                              o["path_len"], self.cap, d["prefix_len"])
+        self.launches_last_step = n_launch + self.ctx.last_launch_count
+        if events_after is not None:
+            events_after.record()           # the device work of this step ends here
         plen = o["path_len"].cpu().numpy()
         nodes = o["path_nodes"].cpu().numpy()
         bonus = self.bonus.cpu().numpy()

@@ -71,3 +71,42 @@ def test_head_is_deterministic_run_to_run():
     a, _, _ = run_head(w, parent, 13)
     b, _, _ = run_head(w, parent, 13)
     assert np.array_equal(a["logits"], b["logits"]) and np.array_equal(a["lse"], b["lse"])
+
+
+def test_logit_space_similarity_and_acceptance():
+    """Appendix B's variant: the cosines of Eq. 1 / Eq. 2 taken between rows of logits instead of hidden
+    states -- cascade_similarity with feat = logits, feat_dim = V -- and the rule run on those scores."""
+    w = synth.workload("mini", B=2)
+    parent = w.parent()
+    T = len(parent)
+    ctx = G.make_ctx(w, T)
+    tree = cb.Tree(ctx, parent)
+    rng = np.random.default_rng(31)
+    E, hidden, gamma, tok, p, u = G.tail_inputs(w, rng, parent)
+    dev = lambda a: torch.from_numpy(a).to(G.DEV)
+    z = lambda *s, dt=torch.float32: torch.zeros(s, dtype=dt, device=G.DEV)
+    logits, feat, fnorm, lse, cp, cg = z(w.B, T, w.V), z(w.B, T, w.h), z(w.B, T), z(w.B, T), z(w.B, T), z(w.B, T)
+    cb.cascade_lm_head_cfg(ctx, tree, G.to_dev(hidden, w.dtype), dev(gamma), w.eps, G.to_dev(E, w.dtype), w.cfg_scale,
+                           1.0, dev(tok), logits, feat, fnorm, lse, cp, cg)
+    scores = z(w.B, max(tree.num_pairs, 1))
+    cb.cascade_similarity(ctx, tree, logits, w.V, None, scores)
+    accept = z(w.B, T, dt=torch.uint8)
+    qR, tvd = z(w.B, T), z(w.B, T)
+    near = z(w.B, dt=torch.int32)
+    prm = cb.Params(w.tau_pos, w.tau_seq, w.tvd_budget, cb.USE_I | cb.USE_C)
+    cb.cascade_relaxed_accept(ctx, tree, scores, None, lse, cp, cg, dev(tok), dev(p), dev(u), prm, accept, qR, tvd, near)
+    nodes, plen, used = z(w.B, tree.depth + 1, dt=torch.int32), z(w.B, dt=torch.int32), z(w.B)
+    cb.cascade_select_path(ctx, tree, accept, tvd, cb.SELECT_LONGEST, nodes, plen, used)
+    torch.cuda.synchronize()
+    ctx.check()
+    lg = logits.cpu().numpy().astype(np.float64)
+    pa, pb = tree.pairs()
+    got = scores.cpu().numpy()
+    for b in range(w.B):
+        ref = np.array([O.cosine(lg[b][a], lg[b][c]) for a, c in zip(pa, pb)])
+        assert np.abs(got[b] - ref).max() < 2e-5
+    rows = [O.relaxed_accept(lg[b], lg[b], tok[b], parent, p[b], u[b], w.tau_pos, w.tau_seq, w.tvd_budget)
+            for b in range(w.B)]
+    G.compare_decisions(parent, rows, accept.cpu().numpy(), nodes.cpu().numpy(), plen.cpu().numpy(), cb.SELECT_LONGEST)
+    tree.close()
+    ctx.close()
