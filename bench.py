@@ -433,7 +433,11 @@ def main():
         "gemm_gate_up": 2 * w.ffn * w.h * e + act * w.h,
         "gemm_down": w.h * w.ffn * e + act * w.ffn,
     }
-    alg_f = {"gemm_head": 2.0 * w.B * T * w.h * w.V}
+    # algorithmic flops: the head's guidance mix is taken before the product (half of two heads); the layer
+    # projections work on both rows of every prompt
+    M2 = R * T
+    alg_f = {"gemm_head": 2.0 * w.B * T * w.h * w.V, "gemm_qkv": 2.0 * M2 * w.h * 3 * hd, "gemm_o": 2.0 * M2 * hd * w.h,
+             "gemm_gate_up": 2.0 * M2 * w.h * 2 * w.ffn, "gemm_down": 2.0 * M2 * w.ffn * w.h}
     per_kernel = {k: {"us": 1e3 * v[0] / v[1], "launches_per_step": v[1] / kt_steps} for k, v in timing.items()}
     step_us_kernels = sum(1e3 * v[0] for v in timing.values()) / kt_steps
     dom = max((k for k in timing if k in alg_b), key=lambda k: timing[k][0])
@@ -461,6 +465,13 @@ def main():
         if k in alg_f:
             d["tensor_tflops"] = alg_f[k] / (us * 1e-6) / 1e12
             d["tensor_frac_of_bf16_peak"] = d["tensor_tflops"] / peaks["bf16_tflops"]
+            # the operand is a bf16 pair (value + remainder): twice the algorithmic tensor work is executed
+            d["executed_tflops"] = 2 * d["tensor_tflops"]
+            if alg_f[k] / (peaks["bf16_tflops"] * 1e12) > alg_b[k] / (peaks["hbm_gbs"] * 1e9):
+                # more rows than the ridge: the tensor cores bound this launch, not the weight stream
+                d.update({"bound": "tensor", "achieved": d["tensor_tflops"], "peak": peaks["bf16_tflops"],
+                          "unit": "TFLOP/s", "frac": d["tensor_frac_of_bf16_peak"],
+                          "hbm_gbs": ach, "hbm_frac": ach / peaks["hbm_gbs"]})
         return d
     roofline = roof(dom)
     extra = {k: roof(k) for k in per_kernel if k in alg_b and k != dom}
