@@ -111,6 +111,25 @@ def test_ties_and_degenerate_rows():
     assert np.array_equal(once, twice) and np.array_equal(c1, c2)
 
 
+def test_long_rows_at_an_unaligned_address():
+    """Rows longer than the register path holds, starting 4 bytes off a 16-byte boundary: the scalar loads."""
+    V, n = 16384 + 1000, 3
+    rng = np.random.default_rng(77)
+    logits = cluster_logits(rng, n, V)
+    w = synth.workload("mini", B=1, V=V)
+    ctx = G.make_ctx(w, 64)
+    buf = torch.zeros(n * V + 4, device=G.DEV)
+    view = buf[1:1 + n * V].view(n, V)
+    view.copy_(torch.from_numpy(logits))
+    assert view.data_ptr() % 16 == 4
+    cnt = torch.zeros(n, dtype=torch.int32, device=G.DEV)
+    cb.cascade_filter_logits(ctx, view, 300, 0.9, cnt)
+    torch.cuda.synchronize()
+    ctx.check()
+    check(logits, view.cpu().numpy(), cnt.cpu().numpy(), 300, 0.9)
+    ctx.close()
+
+
 def test_off_settings_and_errors():
     V = 1024
     logits = cluster_logits(np.random.default_rng(9), 4, V)
