@@ -265,7 +265,7 @@ class Workload:
     n_clusters: int
     sigma: float
     prefix_len: int
-    tree: str  # "binary3" | "topk<N>" | "chain<N>"
+    tree: str  # "binary3" | "topk<N>" | "chain<N>" | "nary<b>x<l>"
     cfg_scale: float
     tau_pos: float
     tau_seq: float
@@ -283,6 +283,9 @@ class Workload:
             return static_topk_tree(int(self.tree[4:]))
         if self.tree.startswith("chain"):
             return chain_tree(int(self.tree[5:]))
+        if self.tree.startswith("nary"):           # "nary<b>x<l>": complete tree, b children per node, l draft levels
+            b, l = self.tree[4:].split("x")
+            return complete_tree(int(b), int(l))
         raise ValueError(self.tree)
 
 

@@ -106,3 +106,21 @@ def test_step_refuses_bad_arguments():
     st.select_mode = 7
     assert L.cascade_verify_step(wl.ctx.handle, wl.tree.handle, C.byref(st), None) == cb.ERR_INVALID_ARG
     wl.close()
+
+
+@pytest.mark.parametrize("tree", [
+    "chain0",        # the root alone: nothing drafted, the path is the root
+    "nary32x1",      # one sibling group of the maximum width (496 sibling pairs)
+    "nary2x7",       # 255 rows, seven levels: the row limit of a tree is 256
+    "nary15x2",      # 241 rows, 1680 sibling pairs + 240 edges
+])
+def test_degenerate_and_maximal_trees(tree):
+    w = synth.workload("mini", B=2, tree=tree, prefix_len=70)
+    for mode in (cb.SELECT_LONGEST, cb.SELECT_FIRST_ACCEPT):
+        wl = PiecesWorkload(w, n_sets=1, keep_logits=True, select_mode=mode, flags=cb.USE_I | cb.USE_C)
+        s = wl.run(0)
+        st, agree, rows = check_step(wl, s, mode, cb.USE_I | cb.USE_C)
+        assert st["prompts"] == w.B
+        if tree == "chain0":
+            assert s.out["path_len"].cpu().tolist() == [0, 0] and s.out["accept"].cpu().numpy().all()
+        wl.close()
