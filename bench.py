@@ -55,6 +55,22 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(x: float, device=None) -> float:
+    """The slowest rank's time: N replicas have finished a step when the last of them has."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(steps_per_rank: int, world: int, seconds: float) -> float:
+    """Steps per second of the whole job: every rank ran `steps_per_rank` steps of its own replica."""
+    return world * steps_per_rank / seconds
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed regions run."""
 
@@ -217,17 +233,15 @@ def run_loop(args, dev, peaks, rank, world):
     clocks = sampler.stop()
     dev_ms = sum(a.elapsed_time(b) for a, b in ev)
     launches = loop.launches_last_step * K
-    if world > 1:
-        t = torch.tensor([dev_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dev_ms = float(t.item())
+    dev_ms = max_over_ranks(dev_ms, dev)
+    wall = max_over_ranks(wall, dev)
     loop.close()
     if rank != 0:
         return
     hd = w.n_heads * w.head_dim
     layer_bytes = (4 * hd * w.h + 3 * w.ffn * w.h) * 2
     step_bytes = args.layers * layer_bytes + w.V * w.h * 2
-    value = world * K / (dev_ms * 1e-3)
+    value = whole_job_rate(K, world, dev_ms * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -239,7 +253,7 @@ def run_loop(args, dev, peaks, rank, world):
                    "parallelism": "replicas" if world > 1 else "single"},
         "accepted_tokens_per_step": accepted / (K * w.B), "tokens_per_step_with_bonus": accepted / (K * w.B) + 1,
         "tokens_per_s": value * (accepted / (K * w.B) + 1),
-        "e2e": {"value": world * K / wall, "unit": UNIT, "h2d_bytes_per_step": 3 * w.B * loop.T * 4 + 4 * w.B,
+        "e2e": {"value": whole_job_rate(K, world, wall), "unit": UNIT, "h2d_bytes_per_step": 3 * w.B * loop.T * 4 + 4 * w.B,
                 "d2h_bytes_per_step": w.B * (loop.tree.depth + 1) * 4 + 8 * w.B,
                 "note": "wall clock per step including the host drafter, the copies of its output and the read-back of path and token"},
         "gpu_launches": launches,
@@ -346,11 +360,8 @@ def main():
         e1.record(stream)
         barrier()
         ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        value = world * done / (ms * 1e-3)
+        ms = max_over_ranks(ms, dev)
+        value = whole_job_rate(done, world, ms * 1e-3)
 
         # per-kernel durations, measured live with CUDA events on the launching stream (no graph)
         wl.ctx.timing_enable(True)
@@ -408,10 +419,7 @@ def main():
                                         h_len)
             alpha_sum += int(h_len.sum())
         e2e_s = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([e2e_s], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, dev)
         wl.ctx.check()
 
     if rank != 0:
@@ -493,7 +501,7 @@ def main():
                    "l2": f"inputs rotate over {n_sets} sets of {per_set / 1e6:.0f} MB (> 126 MB L2 between reuses)",
                    "cuda_graph": graph is not None, "parallelism": "replicas" if world > 1 else "single"},
         "accepted_tokens_per_step": alpha_sum / (e2e_steps * w.B),
-        "e2e": {"value": world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": {"value": whole_job_rate(e2e_steps, world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * done,
         "filter_logits": filter_info,
         "launches_per_step": launches_per_step,
