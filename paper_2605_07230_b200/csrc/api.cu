@@ -83,7 +83,11 @@ int64_t carve(cascade_ctx* c, char* base) {
     int64_t need = 0;
     const int shapes[4][2] = {{(s.Hq + 2 * s.Hkv) * s.D, s.h}, {s.h, s.Hq * s.D}, {2 * s.ffn, s.h}, {s.h, s.ffn}};
     for (const auto& nk : shapes) {
-      const int S = s.dtype == CASCADE_BF16 ? gemm_tc_pick_splits(c->sm_count, (int)RT, nk[0], nk[1], c->layer_max_splits) : 1;
+      int S = s.dtype == CASCADE_BF16 ? gemm_tc_pick_splits(c->sm_count, (int)RT, nk[0], nk[1], c->layer_max_splits) : 1;
+      if (s.dtype == CASCADE_BF16) {  // the balanced mode of the gate/up projection may cut a tile once more
+        const SliceMap map = gemm_tc_balanced_map(c, (int)RT, nk[0], nk[1]);
+        if (map.balanced && map.n_slices > S && map.n_slices <= c->layer_max_splits) S = map.n_slices;
+      }
       const int64_t f = (int64_t)S * RT * nk[0];
       if (f > need) need = f;
     }

@@ -60,6 +60,7 @@ struct GemmArgs {
   int unit_q, unit_r;      // units = grid * unit_q + unit_r: CTA c starts at unit c * unit_q + min(c, unit_r)
   int n_tiles;
   int splits;              // 0: contiguous ranges with in-kernel hand-off; S >= 1: S K slices per tile
+  int balanced;            // 1: contiguous ranges, every piece of a tile to its own output matrix (no hand-off)
   long long slice_stride;  // floats between the C matrices of consecutive K slices
   GemmEpilogue epi;
   float* sk_scratch;       // [grid][halves][NB][128] partial accumulators of split tiles
@@ -99,7 +100,10 @@ __device__ __forceinline__ int range_begin(const GemmArgs& p, int c) { return c 
 struct SegmentWalk {
   int u, u_end;
   int n_kb, splits, w, n_items;
-  __device__ SegmentWalk(const GemmArgs& p) : n_kb(p.n_kb), splits(p.splits) {
+  int first_q, first_r;  // balanced mode: for the number of a piece within its tile
+  __device__ SegmentWalk(const GemmArgs& p) : n_kb(p.n_kb), splits(p.balanced ? 0 : p.splits) {
+    first_q = p.balanced ? p.unit_q : 0;
+    first_r = p.unit_r;
     u = range_begin(p, blockIdx.x);
     u_end = range_begin(p, blockIdx.x + 1);
     w = blockIdx.x;
@@ -116,8 +120,12 @@ struct SegmentWalk {
       return true;
     }
     if (u >= u_end) return false;
-    s.slice = 0;
     s.tile = u / n_kb;
+    s.slice = 0;
+    if (first_q > 0) {  // this CTA's index minus the index of the CTA that holds the tile's first K block
+      const int u0 = s.tile * n_kb, big = first_r * (first_q + 1);
+      s.slice = (int)blockIdx.x - (u0 < big ? u0 / (first_q + 1) : first_r + (u0 - big) / first_q);
+    }
     s.kb0 = u - s.tile * n_kb;
     const int left = u_end - u;
     s.kb1 = left < n_kb - s.kb0 ? s.kb0 + left : n_kb;
@@ -540,6 +548,34 @@ int64_t gemm_tc_scratch_floats(int sm_count) { return (int64_t)sm_count * 2 * 12
 // hand-off between CTAs, so TMEM need not hold a third accumulator set, and its matrices have many tiles).
 static int pick_halves(int NB, bool sliced) { return (sliced && NB > 64 && 4 * NB <= 512) ? 2 : 1; }
 
+SliceMap gemm_tc_balanced_map(const cascade_ctx* ctx, int M, int N, int K) {
+  SliceMap map;
+  const OperandLayout lay = operand_layout(M, K);
+  if (lay.n_chunks != 1 || K % kSpan != 0) return map;
+  const int halves = pick_halves(lay.NB, true);
+  const int n_tiles = cascade_detail::ceil_div(N, halves * kTileN);
+  const int n_kb = K / kSpan;  // sliced launches with more than 64 rows carry one span per stage
+  if (halves != 2) return map;
+  const long long units = (long long)n_tiles * n_kb;
+  const int grid = units < ctx->sm_count ? (int)units : ctx->sm_count;
+  map.q = (int)(units / grid);
+  map.r = (int)(units % grid);
+  map.n_kb = n_kb;
+  map.tile_cols = halves * kTileN;
+  int most = 1;
+  for (int t = 0; t < n_tiles; ++t) {
+    auto cta_of = [&](long long u) {
+      const long long big = (long long)map.r * (map.q + 1);
+      return (int)(u < big ? u / (map.q + 1) : map.r + (u - big) / map.q);
+    };
+    const int pieces = cta_of((long long)(t + 1) * n_kb - 1) - cta_of((long long)t * n_kb) + 1;
+    if (pieces > most) most = pieces;
+  }
+  map.n_slices = most;
+  map.balanced = 1;
+  return map;
+}
+
 int gemm_tc_pick_splits(int sm_count, int M, int N, int K, int max_splits) {
   const OperandLayout lay = operand_layout(M, K);
   const int halves = pick_halves(lay.NB, true);
@@ -602,6 +638,9 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   a.units = (long long)n_tiles * a.n_kb;
   a.n_tiles = n_tiles;
   a.splits = epi.splits;
+  a.balanced = epi.balanced;
+  if (epi.balanced && (epi.splits < 1 || a.n_mchunks != 1 || epi.part != nullptr || epi.accumulate || epi.C == nullptr))
+    return CASCADE_ERR_INVALID_ARG;
   a.slice_stride = epi.slice_stride;
   a.stash = epi.splits == 0 && 3 * halves * a.NB <= 512;
   a.tmem_cols = 32;
@@ -618,7 +657,7 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     configured_smem[kern_i] = smem;
   }
-  long long grid = epi.splits > 0 ? (long long)n_tiles * epi.splits : a.units;
+  long long grid = (epi.splits > 0 && !epi.balanced) ? (long long)n_tiles * epi.splits : a.units;
   if (grid > ctx->sm_count) grid = ctx->sm_count;
   // the kernel's work assignment is 32-bit
   if (a.units >= (1ll << 30) || (long long)a.n_kb * (epi.splits + 1) >= (1ll << 30) || (long long)n_tiles * (epi.splits + 1) >= (1ll << 30))

@@ -191,17 +191,33 @@ __global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restr
 
 // act = silu(gate) * up from the slices of the fused gate/up projection ([.., 2*ffn]: gate then up).
 // ffn is a multiple of 4.
-__global__ void __launch_bounds__(kRowThreads) k_swiglu(const float* __restrict__ slices, int n_slices,
+__global__ void __launch_bounds__(kRowThreads) k_swiglu(const float* __restrict__ slices, const SliceMap map,
                                                         long long slice_stride, int ffn,
                                                         __nv_bfloat16* __restrict__ a_op, const OperandLayout lay,
                                                         float* __restrict__ a_f32) {
   const size_t m = blockIdx.y;
+  // pieces per projection tile for the (at most kCntTiles) tiles this CTA's gate and up columns fall into
+  constexpr int kCntTiles = 16;
+  __shared__ int s_cnt[2][kCntTiles];
+  const int col0 = blockIdx.x * kRowThreads * 4;
+  const int t0g = map.balanced ? col0 / map.tile_cols : 0, t0u = map.balanced ? (ffn + col0) / map.tile_cols : 0;
+  if (map.balanced) {
+    if (threadIdx.x < 2 * kCntTiles) {
+      const int which = threadIdx.x / kCntTiles, i = threadIdx.x % kCntTiles;
+      s_cnt[which][i] = slice_count(map, ((which ? t0u : t0g) + i) * map.tile_cols);
+    }
+    __syncthreads();
+  }
   for (int c = blockIdx.x * kRowThreads + threadIdx.x; c < ffn / 4; c += gridDim.x * kRowThreads) {
     float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-    for (int s = 0; s < n_slices; ++s) {
+    // the gate and the up column lie in different tiles of the projection, which may have been cut into
+    // different numbers of pieces (looked up in the table the first threads made)
+    const int n_g = map.balanced ? s_cnt[0][(4 * c) / map.tile_cols - t0g] : map.n_slices;
+    const int n_u = map.balanced ? s_cnt[1][(ffn + 4 * c) / map.tile_cols - t0u] : map.n_slices;
+    for (int s = 0; s < max(n_g, n_u); ++s) {  // one loop: the gate and up loads of a slice go out together
       const float* row = slices + (size_t)s * slice_stride + m * 2 * ffn;
-      add4(g, load4(row + 4 * c));
-      add4(u, load4(row + ffn + 4 * c));
+      if (s < n_g) add4(g, load4(row + 4 * c));
+      if (s < n_u) add4(u, load4(row + ffn + 4 * c));
     }
     put_operand4(a_op, lay, a_f32, ffn, (int)m, 4 * c,
                  make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
@@ -228,16 +244,30 @@ __global__ void __launch_bounds__(256) k_gemm_f32(const float* __restrict__ A, c
 struct Projection {
   int n_slices;
   long long slice_stride;
+  SliceMap map;  // which of the n_slices matrices hold a given column (all of them unless map.balanced)
 };
 
 // out slices = operand x W^T for one weight matrix (or several stacked in memory).
 int project(cascade_ctx* ctx, const void* W, int N, int K, int M, bool operand_is_attn, int kernel_id, Projection* pr,
-            cudaStream_t s) {
+            cudaStream_t s, bool consumer_reads_map = false) {
   pr->slice_stride = (long long)M * N;
+  pr->map = SliceMap{};
   if (ctx->shape.dtype == CASCADE_BF16) {
-    const int S = gemm_tc_pick_splits(ctx->sm_count, M, N, K, ctx->layer_max_splits);
-    pr->n_slices = S;
+    int S = gemm_tc_pick_splits(ctx->sm_count, M, N, K, ctx->layer_max_splits);
     GemmEpilogue e;
+    if (consumer_reads_map) {
+      // equal ranges of (tile, K block) units per CTA instead of whole (tile, slice) items: no CTA is left with
+      // one item while the others have two
+      const SliceMap map = gemm_tc_balanced_map(ctx, M, N, K);
+      if (map.balanced && map.n_slices <= ctx->layer_max_splits &&
+          (long long)map.n_slices * M * N <= ctx->gemm_out_floats) {
+        pr->map = map;
+        S = map.n_slices;
+        e.balanced = 1;
+      }
+    }
+    pr->n_slices = S;
+    pr->map.n_slices = S;
     e.C = ctx->gemm_out;
     e.ldc = N;
     e.splits = S;
@@ -248,6 +278,7 @@ int project(cascade_ctx* ctx, const void* W, int N, int K, int M, bool operand_i
                           operand_is_attn ? (const __nv_bfloat16*)ctx->attn_out : ctx->act, M, e, kernel_id, s);
   }
   pr->n_slices = 1;
+  pr->map.n_slices = 1;
   dim3 grid(cascade_detail::ceil_div(N, 8), cascade_detail::ceil_div(M, 8));
   {
     KernelScope ks(ctx, K_GEMM_F32, s);
@@ -322,12 +353,12 @@ int run_layers_t(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step*
     CASCADE_TRY(resid_norm<E>(ctx, T, nullptr, nullptr, &pr, L.gamma_mlp, st->eps, nullptr, K_RESID_NORM, s));
     // gate and up stacked in memory: one projection
     if ((const char*)L.w_up != (const char*)L.w_gate + (size_t)sh.ffn * sh.h * es) return CASCADE_ERR_UNSUPPORTED_SHAPE;
-    CASCADE_TRY(project(ctx, L.w_gate, 2 * sh.ffn, sh.h, M, false, K_GEMM_GATE_UP, &pr, s));
+    CASCADE_TRY(project(ctx, L.w_gate, 2 * sh.ffn, sh.h, M, false, K_GEMM_GATE_UP, &pr, s, true));
     {
       const bool bf16 = sh.dtype == CASCADE_BF16;
       KernelScope ks(ctx, K_SWIGLU, s);
       k_swiglu<<<dim3(cascade_detail::ceil_div(sh.ffn / 4, kRowThreads), M), kRowThreads, 0, s>>>(
-          ctx->gemm_out, pr.n_slices, pr.slice_stride, sh.ffn, bf16 ? ctx->act : nullptr, operand_layout(M, sh.ffn),
+          ctx->gemm_out, pr.map, pr.slice_stride, sh.ffn, bf16 ? ctx->act : nullptr, operand_layout(M, sh.ffn),
           bf16 ? nullptr : ctx->act_f32);
     }
     CASCADE_CUDA_TRY(cudaGetLastError());
