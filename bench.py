@@ -210,7 +210,7 @@ def run_loop(args, dev, peaks, rank, world):
     from paper_2605_07230_b200 import synth
     from paper_2605_07230_b200.workload import DecodeLoop
 
-    K, W = min(args.steps, 78), 4                      # 64 + 82 * 7 = 638 cache rows: the workload's 64 -> 64 + 576
+    K, W = max(1, min(args.steps, 78)), 4                      # 64 + 82 * 7 = 638 cache rows: the workload's 64 -> 64 + 576
     w = synth.workload("janus", prefix_len=64)
     loop = DecodeLoop(w, n_layers=args.layers, max_steps=K + W, device=dev, seed=5, tile_layers=True)
     for _ in range(W):
@@ -318,7 +318,7 @@ def main():
         wl = LayerWorkload(w, n_layers=1, device=dev, n_sets=n_sets, want_hidden=False)
     else:
         wl = PiecesWorkload(w, device=dev, n_sets=n_sets)
-    K, W = args.steps, max(args.warmup, 3)
+    K, W = max(args.steps, 1), max(args.warmup, 3)
 
     stream = torch.cuda.Stream()
     graph = None
@@ -337,10 +337,13 @@ def main():
             stream.synchronize()
 
         def run_steps(n):
+            # exactly n steps: whole replays of the n_sets-step graph, the remainder enqueued step by step
             if graph is not None:
                 for _ in range(n // n_sets):
                     graph.replay()
-                return (n // n_sets) * n_sets
+                for i in range(n % n_sets):
+                    wl.run(i)
+                return n
             for i in range(n):
                 wl.run(i)
             return n
