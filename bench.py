@@ -279,6 +279,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--top-k", type=int, default=2000,
                     help="also time cascade_filter_logits (top-k truncation of the target logits, outside the step); 0 = skip")
+    ap.add_argument("--truncate", action="store_true",
+                    help="the timed step itself truncates the target distribution to --top-k (logits are then stored)")
     ap.add_argument("--sets", type=int, default=0, help="rotating input sets (0 = enough to exceed the L2 per step)")
     args = ap.parse_args()
 
@@ -315,9 +317,12 @@ def main():
     per_set = (w.V * w.h + 2 * 2 * w.B * (w.prefix_len + T) * hd) * 2 + layer_bytes
     n_sets = args.sets or max(2, int(np.ceil(3 * 126e6 / per_set)))
     if args.mode == "layer":
-        wl = LayerWorkload(w, n_layers=1, device=dev, n_sets=n_sets, want_hidden=False)
+        wl = LayerWorkload(w, n_layers=1, device=dev, n_sets=n_sets, want_hidden=False, keep_logits=args.truncate)
     else:
-        wl = PiecesWorkload(w, device=dev, n_sets=n_sets)
+        wl = PiecesWorkload(w, device=dev, n_sets=n_sets, keep_logits=args.truncate)
+    if args.truncate:
+        for st_ in wl.sets:
+            st_.step.top_k = args.top_k
     K, W = max(args.steps, 1), max(args.warmup, 3)
 
     stream = torch.cuda.Stream()
@@ -497,7 +502,7 @@ def main():
         "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "tree_rows": T, "prefix_len": w.prefix_len, "V": w.V, "h": w.h,
                    "heads": w.n_heads, "head_dim": w.head_dim, "cfg_scale": w.cfg_scale,
-                   "mode": args.mode,
+                   "mode": args.mode, "top_k_in_step": args.top_k if args.truncate else 0,
                    "step": ("embedding + one decoder layer (q/k/v, rotary, tree attention, output projection, SwiGLU MLP) + "
                             if args.mode == "layer" else "") +
                            "tree attention + final norm + LM head/CFG + relaxed acceptance + path selection",

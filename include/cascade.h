@@ -281,6 +281,11 @@ typedef struct {
   float* hidden_out;           /* [R,T,h] float: residual stream entering the final norm (n_layers>0) */
   void* k_tree_out;            /* [n_layers,R,T,Hkv,D] elem: rotated keys / values of the tree rows, */
   void* v_tree_out;            /*   what a caller appends to the cache for the accepted path          */
+  /* truncation of the target distribution before the rule (see cascade_filter_logits; Appendix D.1):
+   * top_k > 0 and/or 0 < top_p < 1 switch it on, which needs `logits` (they are truncated in place and the
+   * row statistics are taken from them); zero in both fields (a zeroed struct): off */
+  int32_t top_k;
+  float top_p;
 } cascade_step;
 
 /* Runs pieces (a)-(d) (and the decoder layers, if any) as one enqueue on `stream`. */

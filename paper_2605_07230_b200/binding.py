@@ -60,6 +60,7 @@ class Step(C.Structure):
         ("tvd_out", C.c_void_p), ("tvd_used", C.c_void_p), ("near_count", C.c_void_p),
         ("logits", C.c_void_p), ("feat", C.c_void_p), ("scores", C.c_void_p), ("row_lse", C.c_void_p),
         ("hidden_out", C.c_void_p), ("k_tree_out", C.c_void_p), ("v_tree_out", C.c_void_p),
+        ("top_k", C.c_int32), ("top_p", C.c_float),
     ]
 
 

@@ -398,8 +398,19 @@ __global__ void __launch_bounds__(256) k_row_stats(const float* __restrict__ log
   const float* l = logits + ((size_t)b * T + row) * V;
   __shared__ float red[8];
   __shared__ float s_max;
+  // 16 bytes per lane where the row allows it (V is a multiple of 8; the base may not be aligned)
+  const bool vec = (reinterpret_cast<uintptr_t>(l) & 15u) == 0 && (V & 3) == 0;
+  const float4* l4 = reinterpret_cast<const float4*>(l);
   float m = -INFINITY;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) m = fmaxf(m, l[i]);
+  if (vec) {
+#pragma unroll 4
+    for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
+      const float4 x = l4[i];
+      m = fmaxf(fmaxf(m, fmaxf(x.x, x.y)), fmaxf(x.z, x.w));
+    }
+  } else {
+    for (int i = threadIdx.x; i < V; i += blockDim.x) m = fmaxf(m, l[i]);
+  }
   m = warp_max(m);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
   __syncthreads();
@@ -411,7 +422,15 @@ __global__ void __launch_bounds__(256) k_row_stats(const float* __restrict__ log
   __syncthreads();
   m = s_max;
   float sum = 0.f;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) sum += expf(l[i] - m);
+  if (vec) {
+#pragma unroll 4
+    for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
+      const float4 x = l4[i];
+      sum += (expf(x.x - m) + expf(x.y - m)) + (expf(x.z - m) + expf(x.w - m));
+    }
+  } else {
+    for (int i = threadIdx.x; i < V; i += blockDim.x) sum += expf(l[i] - m);
+  }
   sum = warp_sum(sum);
   __syncthreads();
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sum;

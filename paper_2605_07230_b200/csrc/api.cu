@@ -528,6 +528,10 @@ static int verify_step_impl(cascade_ctx* ctx, const cascade_tree* tree, const ca
     return CASCADE_ERR_INVALID_ARG;
   if (st->n_layers < 0) return CASCADE_ERR_INVALID_ARG;
   if (st->n_layers == 0 && st->hidden_in == nullptr) return CASCADE_ERR_INVALID_ARG;
+  const bool nucleus = st->top_p > 0.f && st->top_p < 1.f;
+  const bool truncate = (st->top_k > 0 && st->top_k < ctx->shape.V) || nucleus;
+  if (st->top_k < 0 || st->top_p < 0.f || st->top_p > 1.f || st->top_p != st->top_p) return CASCADE_ERR_INVALID_ARG;
+  if (truncate && st->logits == nullptr) return CASCADE_ERR_INVALID_ARG;  // the truncation works on stored logits
   ctx->launches = 0;
   const void* hidden = st->hidden_in;
   PendingAdd pending;
@@ -545,12 +549,19 @@ static int verify_step_impl(cascade_ctx* ctx, const cascade_tree* tree, const ca
                            st->tok, st->logits, feat, ctx->feat_norm, row_lse, ctx->cand_parent, ctx->cand_gparent, false,
                            st->n_layers > 0, pending, s));
   // cosines, row log-sum-exp (bf16: folded from the head's partials), the rule and the path: one launch
+  if (truncate) {
+    // truncate the stored logits, then take every row's log-sum-exp and candidate logits from what is left
+    CASCADE_TRY(launch_filter_logits(ctx, st->logits, ctx->shape.B * tree->T, st->top_k, nucleus ? st->top_p : 1.f,
+                                     nullptr, s));
+    CASCADE_TRY(launch_row_stats_from_logits(ctx, tree, st->logits, st->tok, row_lse, ctx->cand_parent,
+                                             ctx->cand_gparent, s));
+  }
   TailWork w;
   w.feat = feat;
   w.feat_dim = ctx->shape.h;
   w.feat_norm = ctx->feat_norm;
   w.scores = st->scores ? st->scores : ctx->scores;
-  if (bf16) {
+  if (bf16 && !truncate) {
     w.part = ctx->head_part;
     w.part_ld = ctx->head_max_tiles;
     w.n_tiles = ceil_div(ctx->shape.V, 128);

@@ -206,6 +206,10 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
 
 // head.cu (norm + mix producers, fp32 head) / gemm_tc.cu (tcgen05 GEMM)
 // cand_parent / cand_gparent (may be null) are cleared here; the head fills the entries that exist.
+// Top-k / nucleus truncation of n_rows rows of V logits in place (filter.cu); counts the launch it makes.
+int launch_filter_logits(cascade_ctx* ctx, float* logits, int n_rows, int top_k, float top_p, int32_t* kept_count,
+                         cudaStream_t s);
+
 // Output matrices of a sliced projection that still have to be added to the residual stream.
 struct PendingAdd {
   const float* slices = nullptr;  // [n][R*T][h]

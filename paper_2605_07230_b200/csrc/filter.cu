@@ -265,13 +265,8 @@ __global__ void __launch_bounds__(kFilterThreads) k_filter_logits(float* __restr
 
 }  // namespace
 
-extern "C" int cascade_filter_logits(cascade_ctx* ctx, float* logits, int32_t n_rows, int32_t top_k, float top_p,
-                                     int32_t* kept_count, void* stream) {
-  if (ctx == nullptr || logits == nullptr) return CASCADE_ERR_INVALID_ARG;
-  if (n_rows < 1 || top_k < 0 || !(top_p > 0.f) || top_p > 1.f) return CASCADE_ERR_INVALID_ARG;  // also rejects NaN
-  ctx->launches = 0;
-  if ((top_k == 0 || top_k >= ctx->shape.V) && top_p >= 1.f && kept_count == nullptr) return CASCADE_OK;  // nothing to do
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
+int launch_filter_logits(cascade_ctx* ctx, float* logits, int n_rows, int top_k, float top_p, int32_t* kept_count,
+                         cudaStream_t s) {
   const size_t smem = (size_t)kWarps * 256 * sizeof(unsigned long long);  // 64 KB of per-warp histograms
   const bool in_regs = ctx->shape.V <= kRegItems * kFilterThreads;
   static bool configured = false;
@@ -289,4 +284,13 @@ extern "C" int cascade_filter_logits(cascade_ctx* ctx, float* logits, int32_t n_
   }
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
+}
+
+extern "C" int cascade_filter_logits(cascade_ctx* ctx, float* logits, int32_t n_rows, int32_t top_k, float top_p,
+                                     int32_t* kept_count, void* stream) {
+  if (ctx == nullptr || logits == nullptr) return CASCADE_ERR_INVALID_ARG;
+  if (n_rows < 1 || top_k < 0 || !(top_p > 0.f) || top_p > 1.f) return CASCADE_ERR_INVALID_ARG;  // also rejects NaN
+  ctx->launches = 0;
+  if ((top_k == 0 || top_k >= ctx->shape.V) && top_p >= 1.f && kept_count == nullptr) return CASCADE_OK;  // nothing to do
+  return launch_filter_logits(ctx, logits, n_rows, top_k, top_p, kept_count, static_cast<cudaStream_t>(stream));
 }

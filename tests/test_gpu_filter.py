@@ -190,3 +190,47 @@ def test_truncated_target_feeds_acceptance():
     print(f"truncation to top-{top_k}: {dropped} draft tokens outside the kept set, {stats}")
     tree.close()
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", [cb.SELECT_LONGEST, cb.SELECT_FIRST_ACCEPT])
+def test_fused_step_with_truncation(mode):
+    """cascade_verify_step with top_k / top_p set: the stored logits come back truncated as the checker
+    truncates the untruncated ones, and accept bits and paths are the checker's rule on those."""
+    from paper_2605_07230_b200.workload import PiecesWorkload
+    w = synth.workload("mini", B=3, tree="topk60")
+    wl = PiecesWorkload(w, n_sets=1, keep_logits=True, select_mode=mode)
+    s = wl.run(0)
+    torch.cuda.synchronize()
+    wl.ctx.check()
+    raw = s.out["logits"].cpu().numpy().copy()
+    base_launches = wl.ctx.last_launch_count
+    for top_k, top_p in ((w.V // 16, 0.0), (0, 0.9), (w.V // 8, 0.8)):
+        s.step.top_k, s.step.top_p = top_k, top_p
+        wl.run(0)
+        torch.cuda.synchronize()
+        wl.ctx.check()
+        assert wl.ctx.last_launch_count == base_launches + 2          # truncation + row statistics
+        got = s.out["logits"].cpu().numpy()
+        filt, _ = O.filter_logits(raw.astype(np.float64), top_k, top_p if top_p > 0 else 1.0)
+        differ = np.isneginf(filt) != np.isneginf(got)
+        assert differ.sum() <= (2 if top_p > 0 else 0)                 # nucleus: tokens within the band of p
+        if differ.any():
+            continue
+        feat = s.out["feat"].cpu().numpy().astype(np.float64)
+        h = s.host
+        rows = [O.relaxed_accept(feat[b], filt[b], h["tok"][b], wl.parent, h["draft_p"][b], h["uniforms"][b],
+                                 w.tau_pos, w.tau_seq, w.tvd_budget) for b in range(w.B)]
+        G.compare_decisions(wl.parent, rows, s.out["accept"].cpu().numpy(), s.out["path_nodes"].cpu().numpy(),
+                            s.out["path_len"].cpu().numpy(), mode)
+    # the truncation needs stored logits, and its parameters are validated
+    import ctypes as C2
+    s.step.top_k, s.step.top_p = 5, 0.0
+    saved = s.step.logits
+    s.step.logits = None
+    assert cb.lib().cascade_verify_step(wl.ctx.handle, wl.tree.handle, C2.byref(s.step), None) == cb.ERR_INVALID_ARG
+    s.step.logits = saved
+    s.step.top_k, s.step.top_p = -1, 0.0
+    assert cb.lib().cascade_verify_step(wl.ctx.handle, wl.tree.handle, C2.byref(s.step), None) == cb.ERR_INVALID_ARG
+    s.step.top_k, s.step.top_p = 0, 1.5
+    assert cb.lib().cascade_verify_step(wl.ctx.handle, wl.tree.handle, C2.byref(s.step), None) == cb.ERR_INVALID_ARG
+    wl.close()
