@@ -129,3 +129,23 @@ def test_filtered_rows_feed_the_acceptance_rule():
     r = O.relaxed_accept(feat, f, tok, parent, np.array([1.0, 0.5, 0.5]), np.array([0.0, 0.0, 0.0]), 2.0, 2.0, 0.5)
     assert np.isclose(r["q_plain"][1], O.softmax(f[0])[top]) and r["q_plain"][2] == 0.0
     assert r["accept"][1] == 1 and r["accept"][2] == 0
+
+
+def test_hand_computed_row():
+    """softmax([2, 1, 0, -1]) = [0.6439, 0.2369, 0.0871, 0.0321] (e^2 : e : 1 : 1/e over their sum 11.4752)."""
+    l = np.array([[2.0, 1.0, 0.0, -1.0]])
+    z = np.exp(2) + np.exp(1) + 1 + np.exp(-1)
+    p = np.array([np.exp(2), np.exp(1), 1.0, np.exp(-1)]) / z
+    assert np.allclose(p, [0.6439, 0.2369, 0.0871, 0.0321], atol=5e-5)
+    cases = {
+        (2, 1.0): [1, 1, 0, 0],       # the two largest
+        (0, 0.6): [1, 0, 0, 0],       # 0.6439 alone reaches 0.6
+        (0, 0.7): [1, 1, 0, 0],       # 0.6439 < 0.7 <= 0.8808
+        (0, 0.9): [1, 1, 1, 0],       # 0.8808 < 0.9 <= 0.9679
+        (3, 0.7): [1, 1, 0, 0],       # renormalised over three: 0.6652, 0.2447, 0.0900 -> 0.6652 < 0.7 <= 0.9100
+        (2, 0.72): [1, 0, 0, 0],      # renormalised over two: 0.7311 reaches 0.72 alone
+    }
+    for (k, top_p), want in cases.items():
+        f, kept = O.filter_logits(l, k, top_p)
+        assert kept[0].astype(int).tolist() == want, (k, top_p)
+        assert np.isneginf(f[0][~kept[0]]).all()
