@@ -56,6 +56,8 @@ struct GemmArgs {
   const __nv_bfloat16* A;  // activation operand in the staged layout of operand.cuh
   long long a_chunk_elems; // elements of one row chunk of A (all its K blocks)
   int stash;               // 1: TMEM has room for a third accumulator set (partials of split tiles)
+  int combine;             // 1: one UMMA per K step over both parts of the operand (N = 2 NB), parts added in the epilogue
+  int acc_cols;            // TMEM columns of one accumulator set
   long long units;         // n_tiles * n_kb
   int unit_q, unit_r;      // units = grid * unit_q + unit_r: CTA c starts at unit c * unit_q + min(c, unit_r)
   int n_tiles;
@@ -213,7 +215,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
   } else if (warp == 1) {
     // ---------------- UMMA issue ----------------
     if (lane == 0) {
-      const uint32_t idesc = ptx::umma_idesc_bf16(kTileN, p.NB);
+      // combine: the high parts and the remainders of the activation rows are one 2 NB-row operand (the two
+      // blocks are adjacent in a stage), their products land in separate column ranges and meet in the
+      // epilogue: half as many UMMAs, and the weight tile is read from shared memory once per K step
+      const uint32_t idesc = ptx::umma_idesc_bf16(kTileN, p.combine ? 2 * p.NB : p.NB);
+      const bool combine = p.combine != 0;
       const int stages = p.stages;
       const uint32_t lo_off = (uint32_t)(p.NB * kSpan * 2) >> 4;  // descriptor units of 16 bytes
       int s = 0;
@@ -232,7 +238,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
         ++seg_i;
         if (!ptx::mbar_wait(&tmem_empty[acc], aph ^ 1u, abort_flag, p.err)) break;
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * (uint32_t)(kHalves * p.NB);
+        const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.acc_cols;
         uint32_t accumulate = 0;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
           if (live != 0u) {
@@ -254,7 +260,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
               for (int ks = 0; ks < kSpan / 16; ++ks) {
                 // advancing 16 K elements = 32 bytes = 2 descriptor units inside the swizzle span
                 ptx::umma_bf16_if(live, d, wd0 + 2 * ks, ad0 + 2 * ks, idesc, (q | ks) == 0 ? accumulate : 1u);
-                ptx::umma_bf16_if(live, d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
+                if (!combine) ptx::umma_bf16_if(live, d, wd0 + 2 * ks, ad0 + lo_off + 2 * ks, idesc, 1u);
               }
             }
           }
@@ -296,7 +302,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
       int n_contrib = 0;
       bool presummed = false;
       // spare TMEM columns behind the two accumulator sets hold the sum of the other CTAs' partials
-      const uint32_t stash_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(2 * kHalves * NB);
+      const uint32_t stash_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(2 * p.acc_cols);
       if (owner_of_split) {
         // the CTAs after this one whose range starts inside this tile each hold one partial of it
         const int tile_end = (sg.tile + 1) * p.n_kb;
@@ -344,7 +350,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
         const int n_tile = macro * kHalves + half;
         if (n_tile * kTileN >= p.N) break;  // second half of the last work tile lies beyond N
         const int n = n_tile * kTileN + vl;
-        const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (acc * kHalves + half) * (uint32_t)NB;
+        const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * (uint32_t)p.acc_cols + half * (uint32_t)NB;
         // plain result tiles that lie fully inside C with 16-byte aligned rows take the staged store
         const bool wide_store = c_out != nullptr && !contributor && !e.accumulate && e.part == nullptr &&
                                 (e.ldc & 3) == 0 && (n_tile + 1) * kTileN <= p.N &&
@@ -386,6 +392,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
 #pragma unroll
             for (int sub = 0; sub < 4; ++sub)
               if (16 * sub < n_cols) ptx::tmem_ld16(t_addr + c0 + 16 * sub, v + 16 * sub);
+          }
+          if (p.combine) {  // the remainders' products: NB columns further on
+#pragma unroll
+            for (int sub = 0; sub < 4; ++sub)
+              if (16 * sub < n_cols) {
+                float t[16];
+                ptx::tmem_ld16(t_addr + NB + c0 + 16 * sub, t);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[16 * sub + i] += t[i];
+              }
           }
           if (contributor) {
             // partial of a split tile, [column][weight row]: coalesced over the lanes
@@ -642,9 +658,12 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   if (epi.balanced && (epi.splits < 1 || a.n_mchunks != 1 || epi.part != nullptr || epi.accumulate || epi.C == nullptr))
     return CASCADE_ERR_INVALID_ARG;
   a.slice_stride = epi.slice_stride;
-  a.stash = epi.splits == 0 && 3 * halves * a.NB <= 512;
+  // one UMMA over both operand parts where 64 or fewer activation rows leave the room in TMEM
+  a.combine = (halves == 1 && a.NB <= 64) ? 1 : 0;
+  a.acc_cols = a.combine ? 2 * a.NB : halves * a.NB;
+  a.stash = epi.splits == 0 && 2 * a.acc_cols + halves * a.NB <= 512;
   a.tmem_cols = 32;
-  while (a.tmem_cols < (a.stash ? 3 : 2) * halves * a.NB) a.tmem_cols *= 2;
+  while (a.tmem_cols < 2 * a.acc_cols + (a.stash ? halves * a.NB : 0)) a.tmem_cols *= 2;
   const CUtensorMap* tw =
       get_tmap_2d_bf16(ctx, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)(halves * kTileN), kSpan);
   if (tw == nullptr) return CASCADE_ERR_CUDA;
