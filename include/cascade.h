@@ -128,6 +128,14 @@ const char* cascade_kernel_name(int32_t id);
  * unordered sibling pair).  Returns CASCADE_ERR_BAD_TREE if the ordering rules do not hold. */
 int cascade_tree_create(cascade_ctx* ctx, int32_t T, const int32_t* parent, cascade_tree** out);
 int cascade_tree_destroy(cascade_tree* tree);
+
+/* A new draft tree in an existing descriptor (drafters that grow a different tree every step): same rules
+ * and errors as cascade_tree_create, T <= the context's T_max.  Nothing is allocated; the descriptor is
+ * rebuilt on the host and copied to the device on `stream` (the source is pageable host memory, so the copy
+ * is staged before the call returns), and calls that use the tree must be enqueued after it on that stream.
+ * An invalid tree returns its error and leaves the descriptor as it was.  Host-side queries
+ * (cascade_tree_rows / depth / num_pairs / pairs) answer for the new tree as soon as the call returns. */
+int cascade_tree_update(cascade_tree* tree, int32_t T, const int32_t* parent, void* stream);
 int32_t cascade_tree_rows(const cascade_tree* tree);      /* T                                     */
 int32_t cascade_tree_depth(const cascade_tree* tree);     /* deepest level                         */
 int32_t cascade_tree_num_pairs(const cascade_tree* tree); /* edges + sibling pairs                 */

@@ -25,7 +25,7 @@ KERNEL_COUNT = 24
 
 EXPORTS = [
     "cascade_create", "cascade_destroy", "cascade_workspace_bytes", "cascade_check", "cascade_last_launch_count",
-    "cascade_strerror", "cascade_timing_enable", "cascade_timing_read", "cascade_kernel_name", "cascade_tree_create", "cascade_tree_destroy", "cascade_tree_rows", "cascade_tree_depth",
+    "cascade_strerror", "cascade_timing_enable", "cascade_timing_read", "cascade_kernel_name", "cascade_tree_create", "cascade_tree_destroy", "cascade_tree_update", "cascade_tree_rows", "cascade_tree_depth",
     "cascade_tree_num_pairs", "cascade_tree_pairs", "cascade_tree_attn", "cascade_lm_head_cfg",
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
     "cascade_verify_step_host", "cascade_accept_static", "cascade_bonus_token", "cascade_kv_append",
@@ -88,6 +88,7 @@ def lib() -> C.CDLL:
         L.cascade_kernel_name.restype = C.c_char_p
         L.cascade_tree_create.argtypes = [vp, C.c_int32, vp, C.POINTER(vp)]
         L.cascade_tree_destroy.argtypes = [vp]
+        L.cascade_tree_update.argtypes = [vp, C.c_int32, vp, vp]
         for f in ("cascade_tree_rows", "cascade_tree_depth", "cascade_tree_num_pairs"):
             getattr(L, f).argtypes = [vp]
         L.cascade_tree_pairs.argtypes = [vp, vp, vp]
@@ -189,6 +190,14 @@ class Tree:
         arr = (C.c_int32 * len(parent))(*[int(x) for x in parent])
         self.handle = C.c_void_p()
         _check(lib().cascade_tree_create(ctx.handle, len(parent), arr, C.byref(self.handle)))
+        self.T = lib().cascade_tree_rows(self.handle)
+        self.depth = lib().cascade_tree_depth(self.handle)
+        self.num_pairs = lib().cascade_tree_num_pairs(self.handle)
+
+    def update(self, parent):
+        """A new tree in the same descriptor (no allocation); enqueued on the current stream."""
+        arr = (C.c_int32 * len(parent))(*[int(x) for x in parent])
+        _check(lib().cascade_tree_update(self.handle, len(parent), arr, _stream()))
         self.T = lib().cascade_tree_rows(self.handle)
         self.depth = lib().cascade_tree_depth(self.handle)
         self.num_pairs = lib().cascade_tree_num_pairs(self.handle)

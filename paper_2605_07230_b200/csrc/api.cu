@@ -252,63 +252,113 @@ int cascade_check(cascade_ctx* ctx, void* stream) {
 
 // ---- tree ---------------------------------------------------------------------------------------------
 
-int cascade_tree_create(cascade_ctx* ctx, int32_t T, const int32_t* parent, cascade_tree** out) {
-  if (ctx == nullptr || parent == nullptr || out == nullptr || T < 1) return CASCADE_ERR_INVALID_ARG;
+// Everything the descriptor holds, built on the host from parent[]; nothing is touched on failure.
+namespace {
+struct HostTree {
+  int T = 0, depth_max = 0, n_pairs = 0;
+  std::vector<int32_t> parent, depth, child_begin, child_count, pair_a, pair_b, sib_base;
+  std::vector<uint64_t> anc;
+};
+
+int build_host_tree(const cascade_ctx* ctx, int32_t T, const int32_t* parent, HostTree* h) {
   if (T > ctx->shape.T_max) return CASCADE_ERR_UNSUPPORTED_SHAPE;
   if (parent[0] != -1) return CASCADE_ERR_BAD_TREE;
-  cascade_tree* t = new (std::nothrow) cascade_tree();
-  if (t == nullptr) return CASCADE_ERR_WORKSPACE;
-  t->ctx = ctx;
-  t->T = T;
-  t->parent.assign(parent, parent + T);
-  t->depth.assign(T, 0);
-  t->child_begin.assign(T, 0);
-  t->child_count.assign(T, 0);
-  t->sib_base.assign(T, 0);
+  h->T = T;
+  h->parent.assign(parent, parent + T);
+  h->depth.assign(T, 0);
+  h->child_begin.assign(T, 0);
+  h->child_count.assign(T, 0);
+  h->sib_base.assign(T, 0);
   for (int j = 1; j < T; ++j) {
     const int p = parent[j];
-    if (p < 0 || p >= j) { delete t; return CASCADE_ERR_BAD_TREE; }
-    t->depth[j] = t->depth[p] + 1;
-    if (t->depth[j] < t->depth[j - 1]) { delete t; return CASCADE_ERR_BAD_TREE; }   // BFS order
-    if (j > 1 && p < parent[j - 1]) { delete t; return CASCADE_ERR_BAD_TREE; }      // groups contiguous
-    if (t->child_count[p] == 0) t->child_begin[p] = j;
-    t->child_count[p]++;
-    if (t->child_count[p] > CASCADE_MAX_CHILDREN) { delete t; return CASCADE_ERR_UNSUPPORTED_SHAPE; }
-    t->depth_max = t->depth[j];
+    if (p < 0 || p >= j) return CASCADE_ERR_BAD_TREE;
+    h->depth[j] = h->depth[p] + 1;
+    if (h->depth[j] < h->depth[j - 1]) return CASCADE_ERR_BAD_TREE;   // BFS order
+    if (j > 1 && p < parent[j - 1]) return CASCADE_ERR_BAD_TREE;      // groups contiguous
+    if (h->child_count[p] == 0) h->child_begin[p] = j;
+    h->child_count[p]++;
+    if (h->child_count[p] > CASCADE_MAX_CHILDREN) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+    h->depth_max = h->depth[j];
   }
   // pair list: edge (parent[j], j) at index j-1, then the sibling pairs of each parent in order
   for (int j = 1; j < T; ++j) {
-    t->pair_a.push_back(parent[j]);
-    t->pair_b.push_back(j);
+    h->pair_a.push_back(parent[j]);
+    h->pair_b.push_back(j);
   }
   for (int p = 0; p < T; ++p) {
-    t->sib_base[p] = (int)t->pair_a.size();
-    const int cb = t->child_begin[p], k = t->child_count[p];
+    h->sib_base[p] = (int)h->pair_a.size();
+    const int cb = h->child_begin[p], k = h->child_count[p];
     for (int x = 0; x < k; ++x)
       for (int y = x + 1; y < k; ++y) {
-        t->pair_a.push_back(cb + x);
-        t->pair_b.push_back(cb + y);
+        h->pair_a.push_back(cb + x);
+        h->pair_b.push_back(cb + y);
       }
   }
-  t->n_pairs = (int)t->pair_a.size();
-  if (t->n_pairs > ctx->max_pairs) { delete t; return CASCADE_ERR_UNSUPPORTED_SHAPE; }
-  std::vector<uint64_t> anc((size_t)T * 4, 0);
+  h->n_pairs = (int)h->pair_a.size();
+  if (h->n_pairs > ctx->max_pairs) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  h->anc.assign((size_t)T * 4, 0);
   for (int j = 0; j < T; ++j)
-    for (int i = j; i >= 0; i = parent[i]) anc[(size_t)j * 4 + (i >> 6)] |= 1ull << (i & 63);
+    for (int i = j; i >= 0; i = parent[i]) h->anc[(size_t)j * 4 + (i >> 6)] |= 1ull << (i & 63);
+  return CASCADE_OK;
+}
 
-  const int64_t n_pairs_alloc = t->n_pairs > 0 ? t->n_pairs : 1;
+// Copies a host descriptor into the tree's device arrays (sized for the context's limits) and takes it over.
+int install_host_tree(cascade_tree* t, HostTree&& h, cudaStream_t s, bool async) {
+  bool ok = true;
+  auto up = [&](void* dst, const void* src, size_t n) {
+    if (n == 0) return;
+    const cudaError_t e = async ? cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, s)
+                                : cudaMemcpy(dst, src, n, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) ok = false;
+  };
+  const int T = h.T;
+  up(t->d_parent, h.parent.data(), sizeof(int32_t) * T);
+  up(t->d_depth, h.depth.data(), sizeof(int32_t) * T);
+  up(t->d_child_begin, h.child_begin.data(), sizeof(int32_t) * T);
+  up(t->d_child_count, h.child_count.data(), sizeof(int32_t) * T);
+  up(t->d_sib_base, h.sib_base.data(), sizeof(int32_t) * T);
+  up(t->d_pair_a, h.pair_a.data(), sizeof(int32_t) * h.n_pairs);
+  up(t->d_pair_b, h.pair_b.data(), sizeof(int32_t) * h.n_pairs);
+  up(t->d_anc, h.anc.data(), sizeof(uint64_t) * h.anc.size());
+  if (!ok) {
+    (void)cudaGetLastError();
+    return CASCADE_ERR_CUDA;
+  }
+  t->T = h.T;
+  t->depth_max = h.depth_max;
+  t->n_pairs = h.n_pairs;
+  t->parent = std::move(h.parent);
+  t->depth = std::move(h.depth);
+  t->child_begin = std::move(h.child_begin);
+  t->child_count = std::move(h.child_count);
+  t->pair_a = std::move(h.pair_a);
+  t->pair_b = std::move(h.pair_b);
+  t->sib_base = std::move(h.sib_base);
+  return CASCADE_OK;
+}
+}  // namespace
+
+int cascade_tree_create(cascade_ctx* ctx, int32_t T, const int32_t* parent, cascade_tree** out) {
+  if (ctx == nullptr || parent == nullptr || out == nullptr || T < 1) return CASCADE_ERR_INVALID_ARG;
+  HostTree h;
+  CASCADE_TRY(build_host_tree(ctx, T, parent, &h));
+  cascade_tree* t = new (std::nothrow) cascade_tree();
+  if (t == nullptr) return CASCADE_ERR_WORKSPACE;
+  t->ctx = ctx;
+  // device arrays sized for the context's limits, so that cascade_tree_update never allocates
+  const int64_t T_cap = ctx->shape.T_max, pairs_cap = ctx->max_pairs > 0 ? ctx->max_pairs : 1;
   Carver cv;
   auto layout = [&](char* base) {
     cv = Carver();
     cv.base = base;
-    cv.take(t->d_parent, T);
-    cv.take(t->d_depth, T);
-    cv.take(t->d_child_begin, T);
-    cv.take(t->d_child_count, T);
-    cv.take(t->d_sib_base, T);
-    cv.take(t->d_pair_a, n_pairs_alloc);
-    cv.take(t->d_pair_b, n_pairs_alloc);
-    cv.take(t->d_anc, (int64_t)T * 4);
+    cv.take(t->d_parent, T_cap);
+    cv.take(t->d_depth, T_cap);
+    cv.take(t->d_child_begin, T_cap);
+    cv.take(t->d_child_count, T_cap);
+    cv.take(t->d_sib_base, T_cap);
+    cv.take(t->d_pair_a, pairs_cap);
+    cv.take(t->d_pair_b, pairs_cap);
+    cv.take(t->d_anc, T_cap * 4);
     return align_up(cv.off, 256);
   };
   const int64_t bytes = layout(nullptr);
@@ -318,26 +368,21 @@ int cascade_tree_create(cascade_ctx* ctx, int32_t T, const int32_t* parent, casc
     return CASCADE_ERR_WORKSPACE;
   }
   layout(t->dev);
-  bool ok = true;
-  auto up = [&](void* dst, const void* src, size_t n) {
-    if (n && cudaMemcpy(dst, src, n, cudaMemcpyHostToDevice) != cudaSuccess) ok = false;
-  };
-  up(t->d_parent, t->parent.data(), sizeof(int32_t) * T);
-  up(t->d_depth, t->depth.data(), sizeof(int32_t) * T);
-  up(t->d_child_begin, t->child_begin.data(), sizeof(int32_t) * T);
-  up(t->d_child_count, t->child_count.data(), sizeof(int32_t) * T);
-  up(t->d_sib_base, t->sib_base.data(), sizeof(int32_t) * T);
-  up(t->d_pair_a, t->pair_a.data(), sizeof(int32_t) * t->n_pairs);
-  up(t->d_pair_b, t->pair_b.data(), sizeof(int32_t) * t->n_pairs);
-  up(t->d_anc, anc.data(), sizeof(uint64_t) * anc.size());
-  if (!ok) {
-    (void)cudaGetLastError();
+  const int rc = install_host_tree(t, std::move(h), nullptr, false);
+  if (rc != CASCADE_OK) {
     cudaFree(t->dev);
     delete t;
-    return CASCADE_ERR_CUDA;
+    return rc;
   }
   *out = t;
   return CASCADE_OK;
+}
+
+int cascade_tree_update(cascade_tree* tree, int32_t T, const int32_t* parent, void* stream) {
+  if (tree == nullptr || parent == nullptr || T < 1) return CASCADE_ERR_INVALID_ARG;
+  HostTree h;
+  CASCADE_TRY(build_host_tree(tree->ctx, T, parent, &h));  // an invalid tree leaves the old one in place
+  return install_host_tree(tree, std::move(h), as_stream(stream), true);
 }
 
 int cascade_tree_destroy(cascade_tree* tree) {
