@@ -299,11 +299,12 @@ typedef struct {
 /* Runs pieces (a)-(d) (and the decoder layers, if any) as one enqueue on `stream`. */
 int cascade_verify_step(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step, void* stream);
 
-/* Same step with the per-step inputs and results in HOST memory (pinned memory makes the copies
- * asynchronous): tok, draft_p, uniforms [B,T] are copied in, accept [B,T], path_nodes [B,depth+1] and
- * path_len [B] are copied back, and the call returns after the stream has been synchronised.  The
- * corresponding pointers inside `step` are ignored (the context's own staging buffers are used);
- * everything else in `step` is read as in cascade_verify_step. */
+/* Same step with the per-step inputs and results in HOST memory (pageable or pinned): tok, draft_p, uniforms
+ * [B,T] are gathered into the context's pinned block and copied to the device in one transfer, accept [B,T],
+ * path_nodes [B,depth+1] and path_len [B] come back in one transfer, and the call returns after the stream
+ * has been synchronised, the results in the caller's arrays.  The corresponding pointers inside `step` are
+ * ignored (the context's own staging buffers are used); everything else in `step` is read as in
+ * cascade_verify_step.  Like all calls on one context, these must not overlap. */
 int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step,
                              const int32_t* tok_host, const float* draft_p_host, const float* uniforms_host,
                              uint8_t* accept_host, int32_t* path_nodes_host, int32_t* path_len_host,

@@ -103,12 +103,10 @@ int64_t carve(cascade_ctx* c, char* base) {
     cv.take(p, s.dtype == CASCADE_BF16 ? operand_elems((int)RT, s.Hq * s.D) * 2 : RT * s.Hq * s.D * es);
     c->attn_out = p;
   }
-  cv.take(c->st_tok, BT);
-  cv.take(c->st_draft_p, BT);
-  cv.take(c->st_uniforms, BT);
-  cv.take(c->st_accept, BT);
-  cv.take(c->st_path_nodes, (int64_t)s.B * (T + 1));
-  cv.take(c->st_path_len, s.B);
+  c->st_in_bytes = 3 * BT * 4;
+  c->st_out_bytes = align_up(BT, 4) + (int64_t)s.B * (T + 1) * 4 + (int64_t)s.B * 4;
+  cv.take(c->st_in, c->st_in_bytes);
+  cv.take(c->st_out, c->st_out_bytes);
   return align_up(cv.off, 256);
 }
 
@@ -207,9 +205,11 @@ int cascade_create(cascade_ctx** out, const cascade_shape* shape) {
   }
   carve(c, c->ws);
   if (cudaMemset(c->ws, 0, (size_t)c->ws_bytes) != cudaSuccess ||
-      cudaMallocHost(&c->host_error, 64) != cudaSuccess) {
+      cudaMallocHost(&c->host_error, 64) != cudaSuccess ||
+      cudaMallocHost(&c->host_stage, (size_t)(c->st_in_bytes + c->st_out_bytes)) != cudaSuccess) {
     (void)cudaGetLastError();
     cudaFree(c->ws);
+    if (c->host_error != nullptr) cudaFreeHost(c->host_error);
     delete c;
     return CASCADE_ERR_CUDA;
   }
@@ -227,6 +227,7 @@ int cascade_destroy(cascade_ctx* ctx) {
   for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
   cudaFree(ctx->ws);
   cudaFreeHost(ctx->host_error);
+  cudaFreeHost(ctx->host_stage);
   free_tmap_cache(ctx);
   delete ctx;
   return CASCADE_OK;
@@ -642,23 +643,30 @@ int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const c
     return CASCADE_ERR_INVALID_ARG;
   cudaStream_t s = as_stream(stream);
   const size_t BT = (size_t)ctx->shape.B * tree->T;
-  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->st_tok, tok_host, BT * 4, cudaMemcpyHostToDevice, s));
-  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->st_draft_p, draft_p_host, BT * 4, cudaMemcpyHostToDevice, s));
-  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->st_uniforms, uniforms_host, BT * 4, cudaMemcpyHostToDevice, s));
+  // The three inputs are a few hundred bytes each: they are gathered into one pinned block and go to the device
+  // with one copy, the three results come back the same way (every small copy costs microseconds on the stream).
+  const size_t in_bytes = 3 * BT * 4;
+  const size_t nodes_bytes = (size_t)ctx->shape.B * (tree->depth_max + 1) * 4, len_bytes = (size_t)ctx->shape.B * 4;
+  const size_t acc_pad = (BT + 3) / 4 * 4, out_bytes = acc_pad + nodes_bytes + len_bytes;
+  char* h_in = ctx->host_stage;
+  char* h_out = ctx->host_stage + ctx->st_in_bytes;
+  std::memcpy(h_in, tok_host, BT * 4);
+  std::memcpy(h_in + BT * 4, draft_p_host, BT * 4);
+  std::memcpy(h_in + 2 * BT * 4, uniforms_host, BT * 4);
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(ctx->st_in, h_in, in_bytes, cudaMemcpyHostToDevice, s));
   cascade_step st = *step;
-  st.tok = ctx->st_tok;
-  st.draft_p = ctx->st_draft_p;
-  st.uniforms = ctx->st_uniforms;
-  st.accept = ctx->st_accept;
-  st.path_nodes = ctx->st_path_nodes;
-  st.path_len = ctx->st_path_len;
+  st.tok = reinterpret_cast<const int32_t*>(ctx->st_in);
+  st.draft_p = reinterpret_cast<const float*>(ctx->st_in + BT * 4);
+  st.uniforms = reinterpret_cast<const float*>(ctx->st_in + 2 * BT * 4);
+  st.accept = reinterpret_cast<uint8_t*>(ctx->st_out);
+  st.path_nodes = reinterpret_cast<int32_t*>(ctx->st_out + acc_pad);
+  st.path_len = reinterpret_cast<int32_t*>(ctx->st_out + acc_pad + nodes_bytes);
   CASCADE_TRY(verify_step_impl(ctx, tree, &st, s));
-  CASCADE_CUDA_TRY(cudaMemcpyAsync(accept_host, ctx->st_accept, BT, cudaMemcpyDeviceToHost, s));
-  CASCADE_CUDA_TRY(cudaMemcpyAsync(path_nodes_host, ctx->st_path_nodes,
-                                   (size_t)ctx->shape.B * (tree->depth_max + 1) * 4, cudaMemcpyDeviceToHost, s));
-  CASCADE_CUDA_TRY(cudaMemcpyAsync(path_len_host, ctx->st_path_len, (size_t)ctx->shape.B * 4,
-                                   cudaMemcpyDeviceToHost, s));
+  CASCADE_CUDA_TRY(cudaMemcpyAsync(h_out, ctx->st_out, out_bytes, cudaMemcpyDeviceToHost, s));
   CASCADE_CUDA_TRY(cudaStreamSynchronize(s));
+  std::memcpy(accept_host, h_out, BT);
+  std::memcpy(path_nodes_host, h_out + acc_pad, nodes_bytes);
+  std::memcpy(path_len_host, h_out + acc_pad + nodes_bytes, len_bytes);
   return CASCADE_OK;
 }
 

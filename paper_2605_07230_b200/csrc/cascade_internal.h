@@ -105,12 +105,12 @@ struct cascade_ctx {
                                  // (R*T x Hq*D, bf16 pair) in the GEMM's staged layout
 
   // staging for the host-buffer entry point
-  int32_t* st_tok = nullptr;
-  float* st_draft_p = nullptr;
-  float* st_uniforms = nullptr;
-  uint8_t* st_accept = nullptr;
-  int32_t* st_path_nodes = nullptr;
-  int32_t* st_path_len = nullptr;
+  // host-buffer entry: one block for the step's inputs (tok | draft_p | uniforms) and one for its results
+  // (accept | path_nodes | path_len), each moved with a single copy through a pinned host block
+  char* st_in = nullptr;
+  char* st_out = nullptr;
+  char* host_stage = nullptr;   // pinned: inputs, then results
+  int64_t st_in_bytes = 0, st_out_bytes = 0;
 };
 
 struct cascade_tree {
