@@ -215,6 +215,8 @@ def run_loop(args, dev, peaks, rank, world):
     loop = DecodeLoop(w, n_layers=args.layers, max_steps=K + W, device=dev, seed=5, tile_layers=True)
     for _ in range(W):
         loop.step()
+    if not args.no_graph:
+        loop.capture()      # note: capturing runs nothing; the caches do not advance
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -249,7 +251,7 @@ def run_loop(args, dev, peaks, rank, world):
         "config": {"workload": "loop", "layers": args.layers, "B": w.B, "tree_rows": loop.T, "prefix_len": "64 -> %d" % int(loop.prefix_len_host[0]),
                    "V": w.V, "h": w.h, "ffn": w.ffn, "heads": w.n_heads, "head_dim": w.head_dim,
                    "step": "verify step through all layers + bonus token + cache append; drafter and read-back on the host, outside the device time",
-                   "l2": "each layer streams its own 405 MB of weights (> 126 MB L2)", "cuda_graph": False,
+                   "l2": "each layer streams its own 405 MB of weights (> 126 MB L2)", "cuda_graph": not args.no_graph,
                    "parallelism": "replicas" if world > 1 else "single"},
         "accepted_tokens_per_step": accepted / (K * w.B), "tokens_per_step_with_bonus": accepted / (K * w.B) + 1,
         "tokens_per_s": value * (accepted / (K * w.B) + 1),

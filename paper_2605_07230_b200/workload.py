@@ -269,6 +269,8 @@ class DecodeLoop:
         self.bonus = torch.zeros(B, dtype=torch.int32, device=device)
         self.mass = torch.zeros(B, device=device)
         self.emitted = [[] for _ in range(B)]
+        self.graph = None
+        self.launches_last_step = 0
 
     def draft(self):
         """Next tree of the stand-in drafter below the pending tokens, plus this step's uniforms."""
@@ -278,13 +280,9 @@ class DecodeLoop:
         ub = self.rng.random(w.B, dtype=np.float32)
         return tok, p, u, ub
 
-    def step(self, drafted=None, events_after=None):
-        tok, p, u, ub = drafted if drafted is not None else self.draft()
+    def _enqueue(self):
+        """The device work of one step: verify, draw the token after the path, append the accepted rows."""
         d, o = self.set.dev, self.set.out
-        d["tok"].copy_(torch.from_numpy(tok))
-        d["draft_p"].copy_(torch.from_numpy(p))
-        d["uniforms"].copy_(torch.from_numpy(u))
-        self.u_bonus.copy_(torch.from_numpy(ub))
         cb.cascade_verify_step(self.ctx, self.tree, self.set.step)
         n_launch = self.ctx.last_launch_count
         cb.cascade_bonus_token(self.ctx, self.tree, o["logits"], d["tok"], o["path_nodes"], o["path_len"], self.u_bonus,
@@ -293,6 +291,30 @@ class DecodeLoop:
         cb.cascade_kv_append(self.ctx, self.tree, self.set.step, o["k_tree_out"], o["v_tree_out"], o["path_nodes"],
                              o["path_len"], self.cap, d["prefix_len"])
         self.launches_last_step = n_launch + self.ctx.last_launch_count
+
+    def capture(self):
+        """Record the step's device work once as a CUDA graph; later steps replay it (all its pointers are
+        fixed, the caches' fill levels live in device memory).  Call after at least one ordinary step."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                self._enqueue()
+        torch.cuda.current_stream().wait_stream(side)
+        self.graph = g
+
+    def step(self, drafted=None, events_after=None):
+        tok, p, u, ub = drafted if drafted is not None else self.draft()
+        d, o = self.set.dev, self.set.out
+        d["tok"].copy_(torch.from_numpy(tok))
+        d["draft_p"].copy_(torch.from_numpy(p))
+        d["uniforms"].copy_(torch.from_numpy(u))
+        self.u_bonus.copy_(torch.from_numpy(ub))
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self._enqueue()
         if events_after is not None:
             events_after.record()           # the device work of this step ends here
         plen = o["path_len"].cpu().numpy()

@@ -15,11 +15,12 @@ from tests import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("over,n_layers,steps", [
-    (dict(B=2, tree="topk32", prefix_len=40), 2, 3),
-    (dict(B=1, tree="topk60", prefix_len=130), 3, 2),
+@pytest.mark.parametrize("over,n_layers,steps,graph_after", [
+    (dict(B=2, tree="topk32", prefix_len=40), 2, 3, None),
+    (dict(B=1, tree="topk60", prefix_len=130), 3, 2, None),
+    (dict(B=2, tree="topk32", prefix_len=40), 2, 4, 1),     # steps after the first replay a recorded CUDA graph
 ])
-def test_decode_loop(over, n_layers, steps):
+def test_decode_loop(over, n_layers, steps, graph_after):
     w = synth.workload("mini", **over)
     loop = DecodeLoop(w, n_layers, max_steps=steps, seed=11)
     B, parent = w.B, loop.parent
@@ -29,6 +30,8 @@ def test_decode_loop(over, n_layers, steps):
     plen = h["prefix_len"].astype(np.int64).copy()
     total_accepted = 0
     for it in range(steps):
+        if graph_after is not None and it == graph_after:
+            loop.capture()
         drafted = loop.draft()
         tok, p, u, ub = drafted
         ref = O.verify_step(h["embed"], h["layers"], h["gamma_final"], h["w_head"], tok, parent, k_cache, v_cache, plen,
