@@ -304,7 +304,10 @@ int cascade_verify_step(cascade_ctx* ctx, const cascade_tree* tree, const cascad
  * path_nodes [B,depth+1] and path_len [B] come back in one transfer, and the call returns after the stream
  * has been synchronised, the results in the caller's arrays.  The corresponding pointers inside `step` are
  * ignored (the context's own staging buffers are used); everything else in `step` is read as in
- * cascade_verify_step.  Like all calls on one context, these must not overlap. */
+ * cascade_verify_step.  Like all calls on one context, these must not overlap.  When the same call (same
+ * step contents, tree and stream) is repeated on a stream that can be recorded (not the legacy default
+ * stream), the library records its copies and launches as a CUDA graph at the second call and replays it
+ * afterwards; results are the same either way. */
 int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const cascade_step* step,
                              const int32_t* tok_host, const float* draft_p_host, const float* uniforms_host,
                              uint8_t* accept_host, int32_t* path_nodes_host, int32_t* path_len_host,

@@ -110,12 +110,23 @@ struct cascade_ctx {
   char* st_in = nullptr;
   char* st_out = nullptr;
   char* host_stage = nullptr;   // pinned: inputs, then results
+  // host-buffer entry: the step recorded as a CUDA graph once the same call has been seen twice
+  struct HostGraph {
+    std::vector<unsigned char> key;
+    cudaGraphExec_t exec = nullptr;
+    int state = 0;     // 0: key seen once, 1: graph ready, -1: recording failed for this key
+    int launches = 0;
+    uint64_t last_use = 0;
+  };
+  std::vector<HostGraph> host_graphs;  // a few entries: callers alternate between a few step structures
+  uint64_t host_graph_clock = 0;
   int64_t st_in_bytes = 0, st_out_bytes = 0;
 };
 
 struct cascade_tree {
   cascade_ctx* ctx = nullptr;
   int T = 0, depth_max = 0, n_pairs = 0;
+  uint64_t version = 0;  // counts cascade_tree_update calls
   std::vector<int32_t> parent, depth, child_begin, child_count, pair_a, pair_b, sib_base;
   // device copies
   char* dev = nullptr;

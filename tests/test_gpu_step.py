@@ -89,6 +89,38 @@ def test_host_entry_matches_device_entry():
     wl.close()
 
 
+def test_host_entry_replays_a_recorded_graph_with_new_inputs():
+    """On a stream of its own the host entry records the repeated call as a CUDA graph (from the second
+    identical call on); every call must still give what the device entry gives for that call's inputs,
+    also when the caller alternates between two step structures."""
+    w = synth.workload("mini", B=2)
+    wl = PiecesWorkload(w, n_sets=2, keep_logits=True)
+    rng = np.random.default_rng(3)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    accept = torch.zeros((w.B, wl.T), dtype=torch.uint8).pin_memory()
+    nodes = torch.zeros((w.B, wl.tree.depth + 1), dtype=torch.int32).pin_memory()
+    plen = torch.zeros(w.B, dtype=torch.int32).pin_memory()
+    side = torch.cuda.Stream()
+    lengths = set()
+    for it in range(8):
+        st = wl.sets[it % 2]
+        u = rng.random((w.B, wl.T), dtype=np.float32)            # new uniforms every call: different decisions
+        tok, p = st.host["tok"], st.host["draft_p"]
+        st.dev["uniforms"].copy_(torch.from_numpy(u))
+        wl.run(it % 2)                                             # device entry on the same inputs
+        torch.cuda.synchronize()
+        want = {k: st.out[k].cpu().numpy().copy() for k in ("accept", "path_nodes", "path_len")}
+        with torch.cuda.stream(side):
+            cb.cascade_verify_step_host(wl.ctx, wl.tree, st.step, pin(tok), pin(p), pin(u), accept, nodes, plen)
+        assert wl.ctx.last_launch_count == 4
+        assert np.array_equal(accept.numpy(), want["accept"]), it
+        assert np.array_equal(nodes.numpy(), want["path_nodes"]) and np.array_equal(plen.numpy(), want["path_len"])
+        lengths.add(tuple(plen.numpy().tolist()))
+    assert len(lengths) > 1                                        # the replays really saw different inputs
+    wl.ctx.check()
+    wl.close()
+
+
 def test_step_refuses_bad_arguments():
     w = synth.workload("mini", B=1)
     wl = PiecesWorkload(w, n_sets=1)
