@@ -215,14 +215,17 @@ __global__ void __launch_bounds__(kFilterThreads) k_filter_logits(float* __restr
   keys.row = row;
   keys.V = V;
   keys.load();
-  // row maximum (the nucleus weights are exp(l - max))
-  uint32_t mk = 0;
-  keys.each([&](uint32_t key, bool valid) { mk = valid ? max(mk, key) : mk; });
-  for (int o = 16; o > 0; o >>= 1) mk = max(mk, __shfl_xor_sync(0xffffffffu, mk, o));
-  if ((threadIdx.x & 31) == 0) sh.redf[threadIdx.x >> 5] = __uint_as_float(mk);
-  __syncthreads();
-  for (int i = 0; i < kWarps; ++i) mk = max(mk, __float_as_uint(sh.redf[i]));
-  const float m = key_value(mk);
+  // row maximum: only the nucleus needs it (its weights are exp(l - max))
+  float m = 0.f;
+  if (top_p < 1.f) {
+    uint32_t mk = 0;
+    keys.each([&](uint32_t key, bool valid) { mk = valid ? max(mk, key) : mk; });
+    for (int o = 16; o > 0; o >>= 1) mk = max(mk, __shfl_xor_sync(0xffffffffu, mk, o));
+    if ((threadIdx.x & 31) == 0) sh.redf[threadIdx.x >> 5] = __uint_as_float(mk);
+    __syncthreads();
+    for (int i = 0; i < kWarps; ++i) mk = max(mk, __float_as_uint(sh.redf[i]));
+    m = key_value(mk);
+  }
 
   uint32_t floor_key = 1u;  // every real key (0 marks an empty slot)
   if (top_k > 0 && top_k < V) floor_key = descend<false, kReg>(keys, m, floor_key, (unsigned long long)top_k, sh, hist);
