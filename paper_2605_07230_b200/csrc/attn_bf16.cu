@@ -56,7 +56,8 @@ constexpr int kPBytes = 128 * kTileKeys * 2;  // 32 KB
 constexpr int kKVTileBytes = kTileKeys * kD * 2;  // 32 KB for K, same for V
 constexpr int kKSlots = 2;     // K tiles in shared memory (a slot is free again once S = Q K^T has read it)
 constexpr int kVSlots = 3;     // V tiles in shared memory (free once O += P V has read it)
-constexpr int kPrefetch = 2;   // tiles requested into the L2 beyond what the shared-memory rings hold
+constexpr int kPrefetch = 0;   // with a ring of n slots, tile i + n - 1 + kPrefetch is requested into the L2 when tile i is
+                               // loaded (measured 0..3 on 20-tile rows: deeper requests delay the loads that are waited for)
 constexpr int kSmemBytes = kQBytes + kPBytes + (kKSlots + kVSlots) * kKVTileBytes + 1024;
 constexpr int kXRow = 132;  // row stride (floats) of the half-merge exchange buffer (16-byte aligned rows)
 constexpr int kORow = 132;  // row stride (floats) of the output staging buffer (16-byte aligned rows)
@@ -152,7 +153,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (warp == 4) {
     // ---------------- TMA producers: lane 0 streams Q and the K tiles, lane 1 the V tiles ----------------
     // The rings hold less than HBM latency x this SM's share of the bandwidth, so tiles further ahead
-    // are also requested into the L2 (each request after the tile load it accompanies: the TMA unit works in order).
+    // are also requested into the L2.
     if (lane < 2 && n > 0) {
       const bool is_v = lane == 1;
       const int slots = is_v ? kVSlots : kKSlots;
@@ -169,8 +170,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       int slot = 0;
       uint32_t ph = 0;
       const uint64_t pol_kv = ptx::l2_evict_first();  // the cache is read once per step
-      for (int i = 0; i < n; ++i) {
-        if (!ptx::mbar_wait(&empty[slot], ph ^ 1u, abort_flag, p.err)) break;
+      auto load_tile = [&](int i) {
         const int tile = tile_begin + i;
         const bool in_prefix = tile < n_ptiles;
         const CUtensorMap* m = is_v ? (in_prefix ? &tm_vp : &tm_vt) : (in_prefix ? &tm_kp : &tm_kt);
@@ -183,17 +183,31 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           slot = 0;
           ph ^= 1u;
         }
-        // and ask the L2 for the tile kPrefetch beyond the ring (one per tile: a burst of requests would
-        // queue in front of the loads the ring is waiting for)
+      };
+      auto prefetch_tile = [&](int t) {
+        const int tile = tile_begin + t;
+        const bool in_prefix = tile < n_ptiles;
+        const CUtensorMap* m = is_v ? (in_prefix ? &tm_vp : &tm_vt) : (in_prefix ? &tm_kp : &tm_kt);
+        const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys;
+        ptx::tma_prefetch_4d(m, 0, hk, key0, r);
+        ptx::tma_prefetch_4d(m, 64, hk, key0, r);
+      };
+      // The TMA unit works in order and a request queues in front of whatever is issued after it, so
+      // requests go out in the order the tiles are needed: the rings' first loads, then the tiles beyond
+      // the rings into the L2 (keys and values alternating: the two lanes run these loops in step), then
+      // with every tile loaded into a freed slot one more tile further ahead.
+      const int n_fill = min(slots, n);
+      for (int i = 0; i < n_fill; ++i) load_tile(i);  // the slots start empty
+      __syncwarp(3u);
+      for (int d = 0; d < kVSlots + kPrefetch - 1; ++d) {
+        const int t = slots + d;
+        if (d < slots + kPrefetch - 1 && t < n) prefetch_tile(t);
+      }
+      for (int i = n_fill; i < n; ++i) {
+        if (!ptx::mbar_wait(&empty[slot], ph ^ 1u, abort_flag, p.err)) break;
+        load_tile(i);
         const int t = i + slots + kPrefetch - 1;
-        if (t < n) {
-          const int tile2 = tile_begin + t;
-          const bool pre2 = tile2 < n_ptiles;
-          const CUtensorMap* m2 = is_v ? (pre2 ? &tm_vp : &tm_vt) : (pre2 ? &tm_kp : &tm_kt);
-          const int key2 = (pre2 ? tile2 : tile2 - n_ptiles) * kTileKeys;
-          ptx::tma_prefetch_4d(m2, 0, hk, key2, r);
-          ptx::tma_prefetch_4d(m2, 64, hk, key2, r);
-        }
+        if (t < n) prefetch_tile(t);
       }
     }
   } else if (warp == 5) {
