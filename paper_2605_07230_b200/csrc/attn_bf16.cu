@@ -306,11 +306,13 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       const int tile = tile_begin + i;
       const bool in_prefix = tile < n_ptiles;
       const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys + khalf * 64;
-      // visibility of this lane's 64 keys as one 64-bit word
+      // visibility of this lane's 64 keys as one 64-bit word (rows beyond T see the prefix like any other:
+      // their query is the zero fill of the tensor map and nothing of theirs is ever stored; that keeps the
+      // test below uniform over a warp)
       uint64_t vis;
       if (in_prefix) {
         const int nvis = P - key0;
-        vis = (j >= p.T || nvis <= 0) ? 0ull : (nvis >= 64 ? ~0ull : ((1ull << nvis) - 1ull));
+        vis = nvis <= 0 ? 0ull : (nvis >= 64 ? ~0ull : ((1ull << nvis) - 1ull));
       } else {
         vis = anc_w[(key0 >> 6) & 3];
       }
@@ -318,12 +320,23 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       ptx::tmem_ld64(tmem_s + lane_addr + (i & 1) * 128 + khalf * 64, sc);
       ptx::tc_fence_before();
       ptx::mbar_arrive(&s_empty[i & 1]);
+      // A tile every row of the warp sees whole (all but the last prefix tile) needs no masking, and with a
+      // positive scale the maximum can be taken before scaling: weight = 2^(s * c - m) in one multiply-add.
+      const bool whole = p.c > 0.f && __all_sync(0xffffffffu, vis == ~0ull);
       float m_tile = -INFINITY;
+      if (whole) {
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int k = 0; k < 64; ++k) {
-        sc[k] = ((vis >> k) & 1ull) ? sc[k] * p.c : -INFINITY;
-        m_tile = fmaxf(m_tile, sc[k]);
+        for (int k = 0; k < 64; ++k) m4[k & 3] = fmaxf(m4[k & 3], sc[k]);
+        m_tile = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * p.c;
+      } else {
+#pragma unroll
+        for (int k = 0; k < 64; ++k) {
+          sc[k] = ((vis >> k) & 1ull) ? sc[k] * p.c : -INFINITY;
+          m_tile = fmaxf(m_tile, sc[k]);
+        }
       }
+      const float mul = whole ? p.c : 1.f;  // the masked path has scaled its scores already
       float alpha = 1.f;  // factor for what this lane has accumulated so far
       if (m_run == -INFINITY) {
         m_run = m_tile;   // nothing accumulated yet (all weights so far were zero)
@@ -336,7 +349,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       uint32_t packed[32];
 #pragma unroll
       for (int k = 0; k < 64; k += 2) {
-        const float p0 = ptx::ex2(sc[k] - m_use), p1 = ptx::ex2(sc[k + 1] - m_use);
+        const float p0 = ptx::ex2(fmaf(sc[k], mul, -m_use)), p1 = ptx::ex2(fmaf(sc[k + 1], mul, -m_use));
         packed[k >> 1] = ptx::pack_bf16x2(p0, p1);
         // sum what the tensor core will actually see (bf16-rounded) so that weights add up to one
         rowsum += __uint_as_float(packed[k >> 1] << 16) + __uint_as_float(packed[k >> 1] & 0xffff0000u);
