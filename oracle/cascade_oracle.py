@@ -18,9 +18,10 @@ textbook causal / decode attention, CFG end points and linearity, closed-form co
 to Algorithm 1 with the relaxation off, an independently written sequential walk of Algorithm 2,
 brute-force path enumeration, threshold monotonicity with an unbounded budget, hand-computed trees,
 the library's top-k and a brute-force nucleus for the truncation of the target distribution.
-`decoder_layer` is pinned only through special cases (zero weights -> identity; the rotary map is
-checked against complex multiplication); the architecture itself comes from the workload definition,
-not from the paper.
+`decoder_layer` (architecture from the workload definition, not from the paper) is pinned against an
+ordinary causal block built from torch's library routines: on a chain with an empty prefix, and on a
+branching tree behind prefixes of two lengths, where every root-to-node path must come out as the last
+token of the plain causal sequence  prefix + path  (position = prefix length + depth, ancestors only).
 """
 from __future__ import annotations
 

@@ -108,3 +108,70 @@ def test_verify_step_composes_the_pieces():
                            w.tvd_budget)
     assert np.array_equal(out["accept"][0]["accept"], acc["accept"])
     assert out["accept"][0]["path"] == O.select_path(acc["accept"], parent, acc["tvd_out"])[0]
+
+
+def _causal_block(x_seq, lw, H, D, eps, base):
+    """A plain causal pre-norm block over a token sequence, positions 0..n-1, in torch (library routines:
+    rms_norm, linear, scaled_dot_product_attention, silu).  Returns (output rows, rotated keys, values)."""
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    n, h = x_seq.shape
+    xt = t(x_seq)
+    a = torch.nn.functional.rms_norm(xt, (h,), t(lw.gamma_attn), eps)
+    qt, kt, vt = (torch.nn.functional.linear(a, t(w)).view(n, H, D) for w in (lw.wq, lw.wk, lw.wv))
+
+    def rot(z):
+        inv = base ** (-torch.arange(0, D, 2, dtype=torch.float64) / D)
+        ang = torch.arange(n, dtype=torch.float64)[:, None] * inv[None]
+        cos, sin = torch.cat([ang.cos(), ang.cos()], -1)[:, None], torch.cat([ang.sin(), ang.sin()], -1)[:, None]
+        return z * cos + torch.cat([-z[..., D // 2:], z[..., : D // 2]], -1) * sin
+
+    qt, kt = rot(qt), rot(kt)
+    att = torch.nn.functional.scaled_dot_product_attention(
+        qt.permute(1, 0, 2), kt.permute(1, 0, 2), vt.permute(1, 0, 2), is_causal=True).permute(1, 0, 2)
+    xt = xt + torch.nn.functional.linear(att.reshape(n, H * D), t(lw.wo))
+    m = torch.nn.functional.rms_norm(xt, (h,), t(lw.gamma_mlp), eps)
+    xt = xt + torch.nn.functional.linear(
+        torch.nn.functional.silu(torch.nn.functional.linear(m, t(lw.w_gate))) * torch.nn.functional.linear(m, t(lw.w_up)),
+        t(lw.w_down))
+    return xt.numpy(), kt.numpy(), vt.numpy()
+
+
+def test_every_root_to_node_path_is_a_causal_sequence_after_the_prefix():
+    """Position rule and masking of the layer on a BRANCHING tree with a NON-EMPTY prefix: tree decoding verifies
+    several continuations of one prefix at once (Section 3), so the layer's output at node j must be what an
+    ordinary causal block gives for the last token of the sequence  prefix tokens + root-to-j path.  The cache
+    rows handed to the layer are the keys / values of the prefix tokens rotated at positions 0..P-1.  Using the
+    row index instead of the depth as the position, dropping the prefix length from it, or letting a row see a
+    non-ancestor each fail this for some node.  The two rows of the pair get prefixes of different lengths."""
+    rng = np.random.default_rng(5)
+    h, H, D, ffn = 16, 2, 8, 24
+    eps, base = 1e-5, 10000.0
+    lw = _layer(rng, h, H, D, ffn, 0.2)
+    lw.gamma_attn = rng.uniform(0.5, 1.5, h).astype(np.float32)
+    lw.gamma_mlp = rng.uniform(0.5, 1.5, h).astype(np.float32)
+    parent = synth.static_topk_tree(11, (3, 2, 2))       # 12 rows, three levels, siblings at every level
+    T = len(parent)
+    depth = synth.tree_depth(parent)
+    assert depth.max() == 3 and any(depth[j] != j for j in range(T))
+    P = [5, 3]
+    Pmax = max(P)
+    x_prefix = [rng.standard_normal((p, h)) for p in P]
+    x_tree = rng.standard_normal((2, T, h))
+    kp, vp = np.zeros((2, Pmax, H, D)), np.zeros((2, Pmax, H, D))
+    for r in range(2):
+        _, k, v = _causal_block(x_prefix[r], lw, H, D, eps, base)
+        kp[r, :P[r]], vp[r, :P[r]] = k, v
+        kp[r, P[r]:], vp[r, P[r]:] = 1e6, -1e6          # rows beyond the prefix length must never be read
+    out, q, k, v = O.decoder_layer(x_tree, lw, kp, vp, P, parent, H, D, eps, base, False)
+    for r in range(2):
+        for j in range(T):
+            path = []
+            i = j
+            while i >= 0:
+                path.append(i)
+                i = parent[i]
+            path.reverse()
+            seq = np.concatenate([x_prefix[r], x_tree[r, path]], 0)
+            want, k_seq, v_seq = _causal_block(seq, lw, H, D, eps, base)
+            assert np.allclose(out[r, j], want[-1], atol=1e-10), (r, j)
+            assert np.allclose(k[r, j], k_seq[-1], atol=1e-11) and np.allclose(v[r, j], v_seq[-1], atol=1e-11)
