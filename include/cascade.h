@@ -108,6 +108,18 @@ int cascade_check(cascade_ctx* ctx, void* stream);
 /* Number of kernels the most recent call on this context enqueued. */
 int cascade_last_launch_count(const cascade_ctx* ctx);
 
+/* Failure detection.  Every wait inside a kernel (on an mbarrier, on another CTA's flag) gives up after a
+ * limit, records it in the context's error word and leaves through the kernel's normal teardown, so a wait
+ * that can never end costs the limit, not the device; cascade_check then returns CASCADE_ERR_TIMEOUT and the
+ * context stays usable.  cascade_set_wait_limit changes the limit for later calls on this context
+ * (nanoseconds, >= 1000; default 2 s).
+ * cascade_wait_probe is a self-test of that path: it enqueues one small kernel whose only CTA waits on a
+ * barrier nothing will ever arrive on (no copy in flight), with the context's limit.  waited_ns (DEVICE
+ * uint32, may be NULL) receives how long the wait lasted.  After the stream has been synchronised,
+ * cascade_check reports CASCADE_ERR_TIMEOUT. */
+int cascade_set_wait_limit(cascade_ctx* ctx, int64_t limit_ns);
+int cascade_wait_probe(cascade_ctx* ctx, uint32_t* waited_ns, void* stream);
+
 const char* cascade_strerror(int status);
 
 /* Per-kernel device timing (measurement aid, off by default).  While enabled, every kernel a call on
@@ -115,7 +127,7 @@ const char* cascade_strerror(int status);
  * cascade_timing_read synchronises those events, ADDS the elapsed milliseconds and launch counts per
  * kernel id into ms_total / launches (HOST arrays of CASCADE_KERNEL_COUNT entries, caller-zeroed) and
  * forgets the recorded events.  cascade_kernel_name(id) names an id (NULL if out of range). */
-#define CASCADE_KERNEL_COUNT 24
+#define CASCADE_KERNEL_COUNT 32
 int cascade_timing_enable(cascade_ctx* ctx, int32_t on);
 int cascade_timing_read(cascade_ctx* ctx, float* ms_total, int32_t* launches);
 const char* cascade_kernel_name(int32_t id);
@@ -241,8 +253,8 @@ typedef struct {
   const void* w_gate;      /* [ffn, h] */
   const void* w_up;        /* [ffn, h] */
   const void* w_down;      /* [h, ffn] */
-  const void* k_prefix;    /* [R, prefix_cap, Hkv, D] this layer's cache */
-  const void* v_prefix;
+  void* k_prefix;          /* [R, prefix_cap, Hkv, D] this layer's cache: read by cascade_verify_step, */
+  void* v_prefix;          /* written (rows at and beyond prefix_len) by cascade_kv_append              */
 } cascade_layer;
 
 /* All arguments of one verification step.  Pointers are device pointers except `layers`, a HOST
@@ -331,8 +343,8 @@ int cascade_bonus_token(cascade_ctx* ctx, const cascade_tree* tree, const float*
  * accepted drafts) to the caches of n_layers layers, for both CFG rows of every prompt, at positions
  * prefix_len[r] .. prefix_len[r] + path_len[b], and adds path_len[b] + 1 to prefix_len[r] (device array,
  * updated in place).  The tree rows were rotated at exactly these positions by cascade_verify_step.
- *   layers: HOST array of n_layers structs; only k_prefix / v_prefix are read, and those caches
- *           ([R, prefix_cap, Hkv, D] elem) are WRITTEN here although the struct declares them const.
+ *   layers: HOST array of n_layers structs; only k_prefix / v_prefix are used, and those caches
+ *           ([R, prefix_cap, Hkv, D] elem) are written here.
  *   k_tree, v_tree [n_layers,R,T,Hkv,D] elem: cascade_step.k_tree_out / v_tree_out of the step.
  * A path that does not fit into prefix_cap is not appended and raises CASCADE_ERR_OVERFLOW at the next
  * cascade_check.  n_layers <= 64. */
@@ -377,9 +389,11 @@ int cascade_filter_logits(cascade_ctx* ctx, float* logits, int32_t n_rows, int32
  *   (feat [B,T,feat_dim] float, 16-byte aligned; feat_norm [B,T] or NULL; row_lse, cand_parent,
  *   cand_gparent [B,T]; tok, draft_p, uniforms [B,T]; outputs accept [B,T], path_nodes [B,depth+1],
  *   path_len [B]; q_relaxed, tvd_out, near_count, tvd_used may be NULL).
- * The call allocates nothing on the device: it copies the tree descriptor into the static array, clears
- * the counters and enqueues one kernel on `stream`.  The first call on a device also looks up the device
- * address of the array (cudaGetSymbolAddress), so make that first call outside any stream capture.
+ * The call allocates nothing on the device: it copies the tree descriptor into the static array (from
+ * temporary host memory that is gone when the call returns), clears the counters and enqueues one kernel on
+ * `stream`.  A stream that is being captured is refused (CASCADE_ERR_INVALID_ARG, nothing is enqueued): the
+ * copies read host memory of this call only.  The first call on a device also looks up the device address of
+ * the array (cudaGetSymbolAddress).
  * All calls on a device share the one array and it keeps the last call's contents: two calls whose
  * work overlaps on the GPU (different streams) race; serialise them. */
 #define CASCADE_STATIC_MAX_PROMPTS 32

@@ -21,7 +21,7 @@ ERR_OVERFLOW = -7
 F32, BF16 = 0, 1
 USE_I, USE_C, CONV_DIST_SELF = 1, 2, 4
 SELECT_LONGEST, SELECT_FIRST_ACCEPT = 0, 1
-KERNEL_COUNT = 24
+KERNEL_COUNT = 32
 
 EXPORTS = [
     "cascade_create", "cascade_destroy", "cascade_workspace_bytes", "cascade_check", "cascade_last_launch_count",
@@ -29,7 +29,7 @@ EXPORTS = [
     "cascade_tree_num_pairs", "cascade_tree_pairs", "cascade_tree_attn", "cascade_lm_head_cfg",
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
     "cascade_verify_step_host", "cascade_accept_static", "cascade_bonus_token", "cascade_kv_append",
-    "cascade_filter_logits",
+    "cascade_filter_logits", "cascade_set_wait_limit", "cascade_wait_probe",
 ]
 
 
@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
         L.cascade_bonus_token.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.cascade_kv_append.argtypes = [vp, vp, C.c_int32, C.POINTER(Layer), vp, vp, vp, vp, C.c_int32, vp, vp]
         L.cascade_filter_logits.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_float, vp, vp]
+        L.cascade_set_wait_limit.argtypes = [vp, C.c_int64]
+        L.cascade_wait_probe.argtypes = [vp, vp, vp]
         _lib = L
     return _lib
 
@@ -164,6 +166,13 @@ class Context:
 
     def check(self) -> None:
         _check(lib().cascade_check(self.handle, _stream()))
+
+    def set_wait_limit(self, limit_ns: int) -> None:
+        _check(lib().cascade_set_wait_limit(self.handle, int(limit_ns)))
+
+    def wait_probe(self, waited_ns=None) -> None:
+        """Enqueues the failure-path self-test (a wait that cannot end); check() raises ERR_TIMEOUT afterwards."""
+        _check(lib().cascade_wait_probe(self.handle, _ptr(waited_ns), _stream()))
 
     def timing_enable(self, on: bool) -> None:
         _check(lib().cascade_timing_enable(self.handle, int(on)))

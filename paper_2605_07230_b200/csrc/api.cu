@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument validation, context and tree descriptors, and the composition of
 // the kernels into the exported calls.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -34,6 +35,13 @@ struct Carver {
 };
 
 int elem_size(const cascade_shape& s) { return s.dtype == CASCADE_BF16 ? 2 : 4; }
+
+// Every state a tree descriptor ever holds gets its own number: a recorded step can be told from a step on a
+// descriptor that was destroyed and re-created at the same address, or updated in place.
+uint64_t next_tree_uid() {
+  static std::atomic<uint64_t> counter{0};
+  return ++counter;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -149,7 +157,7 @@ const char* cascade_kernel_name(int32_t id) {
   static const char* names[] = {"tree_attn", "tree_attn_f32", "final_norm_mix", "gemm_head",
                                 "head_f32", "row_stats", "row_lse", "similarity", "accept", "tail", "select_path",
                                 "embed_norm", "gemm_qkv", "rope_split", "gemm_o", "resid_norm", "gemm_gate_up",
-                                "swiglu", "gemm_down", "gemm_f32", "resid_add", "kv_append", "bonus_token", "filter_logits"};
+                                "swiglu", "gemm_down", "gemm_f32", "resid_add", "kv_append", "bonus_token", "filter_logits", "wait_probe"};
   static_assert(sizeof(names) / sizeof(names[0]) == K_KERNEL_ID_END, "one name per kernel id");
   if (id < 0 || id >= K_KERNEL_ID_END) return nullptr;
   return names[id];
@@ -238,6 +246,12 @@ int cascade_destroy(cascade_ctx* ctx) {
 int64_t cascade_workspace_bytes(const cascade_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
 
 int cascade_last_launch_count(const cascade_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int cascade_set_wait_limit(cascade_ctx* ctx, int64_t limit_ns) {
+  if (ctx == nullptr || limit_ns < 1000) return CASCADE_ERR_INVALID_ARG;
+  ctx->wait_limit_ns = (unsigned long long)limit_ns;
+  return CASCADE_OK;
+}
 
 int cascade_check(cascade_ctx* ctx, void* stream) {
   if (ctx == nullptr) return CASCADE_ERR_INVALID_ARG;
@@ -330,7 +344,7 @@ int install_host_tree(cascade_tree* t, HostTree&& h, cudaStream_t s, bool async)
   t->T = h.T;
   t->depth_max = h.depth_max;
   t->n_pairs = h.n_pairs;
-  t->version++;
+  t->uid = next_tree_uid();
   t->parent = std::move(h.parent);
   t->depth = std::move(h.depth);
   t->child_begin = std::move(h.child_begin);
@@ -391,6 +405,15 @@ int cascade_tree_update(cascade_tree* tree, int32_t T, const int32_t* parent, vo
 
 int cascade_tree_destroy(cascade_tree* tree) {
   if (tree == nullptr) return CASCADE_ERR_INVALID_ARG;
+  // steps recorded by the host-buffer entry point into this descriptor's device arrays
+  if (tree->ctx != nullptr) {
+    auto& graphs = tree->ctx->host_graphs;
+    for (size_t i = graphs.size(); i-- > 0;)
+      if (graphs[i].tree == tree) {
+        if (graphs[i].exec != nullptr) cudaGraphExecDestroy(graphs[i].exec);
+        graphs.erase(graphs.begin() + (long)i);
+      }
+  }
   cudaFree(tree->dev);
   delete tree;
   return CASCADE_OK;
@@ -644,6 +667,7 @@ int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const c
   if (ctx == nullptr || tree == nullptr || step == nullptr || tok_host == nullptr || draft_p_host == nullptr ||
       uniforms_host == nullptr || accept_host == nullptr || path_nodes_host == nullptr || path_len_host == nullptr)
     return CASCADE_ERR_INVALID_ARG;
+  if (tree->ctx != ctx) return CASCADE_ERR_INVALID_ARG;  // also bounds T by the context's T_max (the pinned block's size)
   cudaStream_t s = as_stream(stream);
   const size_t BT = (size_t)ctx->shape.B * tree->T;
   // The three inputs are a few hundred bytes each: they are gathered into one pinned block and go to the device
@@ -682,8 +706,11 @@ int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const c
     };
     const void* tp = tree;
     put(&tp, sizeof(tp));
-    put(&tree->version, sizeof(tree->version));
+    put(&tree->uid, sizeof(tree->uid));
     put(&s, sizeof(s));
+    unsigned long long stream_id = 0;  // a new stream that got a destroyed stream's handle has a new id
+    if (s != nullptr && cudaStreamGetId(s, &stream_id) != cudaSuccess) (void)cudaGetLastError();
+    put(&stream_id, sizeof(stream_id));
     put(&st, sizeof(st));
     if (st.n_layers > 0 && st.layers != nullptr) put(st.layers, sizeof(cascade_layer) * (size_t)st.n_layers);
   }
@@ -707,6 +734,7 @@ int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const c
       *hg = cascade_ctx::HostGraph();
     }
     hg->key = key;
+    hg->tree = tree;
     hg->last_use = ++ctx->host_graph_clock;
     CASCADE_TRY(enqueue());  // first sight of this call: run it directly
   } else if (may_record && hg->state == 1) {

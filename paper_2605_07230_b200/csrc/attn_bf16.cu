@@ -73,6 +73,7 @@ struct AttnArgs {
   float2* part_ml;
   float c;  // softmax_scale * log2(e)
   int* err;
+  unsigned long long wait_ns;  // limit of every bounded wait in the kernel
   unsigned int* unit_done;  // [R * Hq * n_rb] finished-split counters, zero between launches
 };
 
@@ -204,7 +205,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (d < slots + kPrefetch - 1 && t < n) prefetch_tile(t);
       }
       for (int i = n_fill; i < n; ++i) {
-        if (!ptx::mbar_wait(&empty[slot], ph ^ 1u, abort_flag, p.err)) break;
+        if (!ptx::mbar_wait(&empty[slot], ph ^ 1u, abort_flag, p.err, p.wait_ns)) break;
         load_tile(i);
         const int t = i + slots + kPrefetch - 1;
         if (t < n) prefetch_tile(t);
@@ -218,7 +219,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if (lane == 0 && n > 0) {
       const uint32_t idesc_s = ptx::umma_idesc_bf16(128, kTileKeys);
       const uint32_t idesc_o = ptx::umma_idesc_bf16_b_mn(128, kD);
-      bool ok = ptx::mbar_wait(&q_full, 0, abort_flag, p.err);
+      bool ok = ptx::mbar_wait(&q_full, 0, abort_flag, p.err, p.wait_ns);
       int is = 0, ip = 0;             // next S, next PV
       int ks_slot = 0, vs_slot = 0;   // ring positions
       uint32_t k_ph = 0, v_ph = 0;
@@ -272,7 +273,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           if (*abort_flag) break;
           const uint64_t now = ptx::global_timer_ns();
           if (polls == 256u) t_idle = now;
-          if (now - t_idle > ptx::kWaitLimitNs) {
+          if (now - t_idle > p.wait_ns) {
             *abort_flag = 1;
             atomicOr(p.err, 1);
             break;
@@ -301,7 +302,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     constexpr float kLazy = 8.f;
     bool ok = n > 0;
     for (int i = 0; ok && i < n; ++i) {
-      if (!ptx::mbar_wait(&s_full[i & 1], (i >> 1) & 1u, abort_flag, p.err)) { ok = false; break; }
+      if (!ptx::mbar_wait(&s_full[i & 1], (i >> 1) & 1u, abort_flag, p.err, p.wait_ns)) { ok = false; break; }
       ptx::tc_fence_after();
       const int tile = tile_begin + i;
       const bool in_prefix = tile < n_ptiles;
@@ -356,7 +357,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
       if (i >= 1) {
         // PV(i-1) complete: P may be overwritten and O holds tiles 0..i-1
-        if (!ptx::mbar_wait(&o_full, (i - 1) & 1u, abort_flag, p.err)) { ok = false; break; }
+        if (!ptx::mbar_wait(&o_full, (i - 1) & 1u, abort_flag, p.err, p.wait_ns)) { ok = false; break; }
         if (__any_sync(0xffffffffu, alpha != 1.f)) {
           ptx::tc_fence_after();
 #pragma unroll
@@ -382,7 +383,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // every instruction line costs a fetch of its own: loops are rolled and the accumulator is taken from
     // TMEM 16 columns at a time instead of as 128 registers.
     bool have_o = false;
-    if (ok && n > 0) have_o = ptx::mbar_wait(&o_full, (n - 1) & 1u, abort_flag, p.err);
+    if (ok && n > 0) have_o = ptx::mbar_wait(&o_full, (n - 1) & 1u, abort_flag, p.err, p.wait_ns);
     have_o = __all_sync(0xffffffffu, have_o);  // the TMEM loads below are warp-wide
     ptx::tc_fence_after();
     // ---- merge the two key halves of each row (lanes r and r+64), then write ----
@@ -594,6 +595,7 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   a.part_ml = ctx->attn_part_ml;
   a.c = scale * 1.4426950408889634f;
   a.err = ctx->dev_error;
+  a.wait_ns = ctx->wait_limit_ns;
   a.unit_done = ctx->attn_unit_done;
   // KV splits: as many as fit on the SMs at once, never more splits than tiles or than the scratch holds
   const int n_tiles = cascade_detail::ceil_div(prefix_cap, kTileKeys) + cascade_detail::ceil_div(T, kTileKeys);
@@ -624,7 +626,7 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
     mvp = get_tmap_4d_bf16(ctx, vp, dp, sp, bkv);
   }
   if (!mq || !mkt || !mvt || !mkp || !mvp) return CASCADE_ERR_CUDA;
-  static bool configured = false;
+  bool& configured = ctx->attn_configured;
   if (!configured) {
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_tree_attn_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     configured = true;

@@ -35,7 +35,7 @@ enum KernelId : int {
   K_TREE_ATTN = 0, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_GEMM_HEAD, K_HEAD_F32, K_ROW_STATS,
   K_ROW_LSE, K_SIMILARITY, K_ACCEPT, K_TAIL, K_SELECT_PATH, K_EMBED_NORM, K_GEMM_QKV, K_ROPE_SPLIT, K_GEMM_O,
   K_RESID_NORM, K_GEMM_GATE_UP, K_SWIGLU, K_GEMM_DOWN, K_GEMM_F32, K_RESID_ADD, K_KV_APPEND, K_BONUS_TOKEN,
-  K_FILTER_LOGITS, K_KERNEL_ID_END
+  K_FILTER_LOGITS, K_WAIT_PROBE, K_KERNEL_ID_END
 };
 static_assert(K_KERNEL_ID_END <= CASCADE_KERNEL_COUNT, "timing table too small");
 
@@ -60,6 +60,10 @@ struct cascade_ctx {
   int* dev_error = nullptr;  // device error word
   int* host_error = nullptr;  // pinned mirror
   bool timing = false;
+  unsigned long long wait_limit_ns = 2000000000ull;  // limit of every bounded device-side wait (cascade_set_wait_limit)
+  // cudaFuncSetAttribute is per device and a context is bound to one device: what has been set is kept here
+  int gemm_smem_configured[3] = {0, 0, 0};
+  bool attn_configured = false, filter_configured = false;
   std::vector<TimedLaunch> timed;        // event pairs recorded since the last read
   std::vector<cudaEvent_t> event_pool;   // spare events
   void* tmap_cache = nullptr; // TMA tensor maps built so far (tmap.cu)
@@ -113,6 +117,7 @@ struct cascade_ctx {
   // host-buffer entry: the step recorded as a CUDA graph once the same call has been seen twice
   struct HostGraph {
     std::vector<unsigned char> key;
+    const cascade_tree* tree = nullptr;  // the descriptor the recorded kernels read (dropped with it)
     cudaGraphExec_t exec = nullptr;
     int state = 0;     // 0: key seen once, 1: graph ready, -1: recording failed for this key
     int launches = 0;
@@ -126,7 +131,7 @@ struct cascade_ctx {
 struct cascade_tree {
   cascade_ctx* ctx = nullptr;
   int T = 0, depth_max = 0, n_pairs = 0;
-  uint64_t version = 0;  // counts cascade_tree_update calls
+  uint64_t uid = 0;      // process-wide unique number of this descriptor's current contents (new at every update)
   std::vector<int32_t> parent, depth, child_begin, child_count, pair_a, pair_b, sib_base;
   // device copies
   char* dev = nullptr;

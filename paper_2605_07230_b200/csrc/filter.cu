@@ -272,7 +272,7 @@ int launch_filter_logits(cascade_ctx* ctx, float* logits, int n_rows, int top_k,
                          cudaStream_t s) {
   const size_t smem = (size_t)kWarps * 256 * sizeof(unsigned long long);  // 64 KB of per-warp histograms
   const bool in_regs = ctx->shape.V <= kRegItems * kFilterThreads;
-  static bool configured = false;
+  bool& configured = ctx->filter_configured;
   if (!configured) {
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_filter_logits<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_filter_logits<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -68,6 +68,7 @@ struct GemmArgs {
   float* sk_scratch;       // [grid][halves][NB][128] partial accumulators of split tiles
   unsigned int* sk_flags;
   int* err;
+  unsigned long long wait_ns;  // limit of every bounded wait in the kernel
 };
 
 __device__ __forceinline__ void combine_ms(float& m, float& s, float mo, float so) {
@@ -193,7 +194,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
         const int n0 = (sg.tile / n_mchunks) * (kHalves * kTileN);
         const __nv_bfloat16* a_chunk = p.A + (size_t)(sg.tile % n_mchunks) * p.a_chunk_elems;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
-          if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.err)) {
+          if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.err, p.wait_ns)) {
             ok = false;
             break;
           }
@@ -236,13 +237,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
       while (ok && walk.next(sg)) {
         const uint32_t acc = seg_i & 1u, aph = (seg_i >> 1) & 1u;
         ++seg_i;
-        if (!ptx::mbar_wait(&tmem_empty[acc], aph ^ 1u, abort_flag, p.err)) break;
+        if (!ptx::mbar_wait(&tmem_empty[acc], aph ^ 1u, abort_flag, p.err, p.wait_ns)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.acc_cols;
         uint32_t accumulate = 0;
         for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
           if (live != 0u) {
-            if (!ptx::mbar_wait(&full_bar[s], ph, abort_flag, p.err)) {
+            if (!ptx::mbar_wait(&full_bar[s], ph, abort_flag, p.err, p.wait_ns)) {
               ok = false;
               break;
             }
@@ -314,7 +315,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
             const uint64_t t0 = ptx::global_timer_ns();
             uint32_t polls = 0;
             while (ld_acquire(f) == 0u) {
-              if ((++polls & 63u) == 0 && ptx::global_timer_ns() - t0 > ptx::kWaitLimitNs) {
+              if ((++polls & 63u) == 0 && ptx::global_timer_ns() - t0 > p.wait_ns) {
                 *abort_flag = 1;
                 atomicOr(p.err, 1);
                 break;
@@ -343,7 +344,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
           }
         }
       }
-      if (!ptx::mbar_wait(&tmem_full[acc], aph, abort_flag, p.err)) break;
+      if (!ptx::mbar_wait(&tmem_full[acc], aph, abort_flag, p.err, p.wait_ns)) break;
       ptx::tc_fence_after();
 #pragma unroll 1  // run-once code: the second half re-uses the instruction lines of the first
       for (int half = 0; half < kHalves; ++half) {
@@ -635,6 +636,7 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   a.sk_scratch = ctx->gemm_scratch;
   a.sk_flags = ctx->gemm_flags;
   a.err = ctx->dev_error;
+  a.wait_ns = ctx->wait_limit_ns;
   // A stage carries 32 KB of weights where three such stages fit (two K spans of a 128-row tile): the
   // round trip of the single producer / issue threads per stage limits the stream below that.  With
   // many activation rows the activation part of a stage is too large for that: one span per stage.
@@ -670,7 +672,7 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   const int smem = a.stages * stage_bytes + 1024;
   if (halves == 2 && spans == 2) return CASCADE_ERR_UNSUPPORTED_SHAPE;  // cannot happen: such stages do not fit
   auto kern = halves == 2 ? k_gemm_tc<2, 1> : (spans == 2 ? k_gemm_tc<1, 2> : k_gemm_tc<1, 1>);
-  static int configured_smem[3] = {0, 0, 0};
+  int* configured_smem = ctx->gemm_smem_configured;
   const int kern_i = halves == 2 ? 2 : spans - 1;
   if (smem > configured_smem[kern_i]) {
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));

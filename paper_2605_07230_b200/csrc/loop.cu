@@ -154,8 +154,8 @@ int cascade_kv_append(cascade_ctx* ctx, const cascade_tree* tree, int32_t n_laye
   for (int i = 0; i < n_layers; ++i) {
     if (layers[i].k_prefix == nullptr || layers[i].v_prefix == nullptr) return CASCADE_ERR_INVALID_ARG;
     if (((uintptr_t)layers[i].k_prefix | (uintptr_t)layers[i].v_prefix) & 15u) return CASCADE_ERR_INVALID_ARG;
-    cp.k[i] = const_cast<void*>(layers[i].k_prefix);
-    cp.v[i] = const_cast<void*>(layers[i].v_prefix);
+    cp.k[i] = layers[i].k_prefix;
+    cp.v[i] = layers[i].v_prefix;
   }
   if (((uintptr_t)k_tree | (uintptr_t)v_tree) & 15u) return CASCADE_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

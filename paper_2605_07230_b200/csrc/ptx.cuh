@@ -64,10 +64,10 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 
 // Bounded wait: gives up after `limit_ns` (checked every 256 failed polls), sets bit 0 of *err_word and
 // the CTA's abort flag, and returns false.  Callers stop issuing work and fall through to the
-// kernel's normal teardown.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+// kernel's normal teardown.  The limit comes from the context (kDefaultWaitLimitNs unless the caller set one).
+constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;  // 2 s
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int* err_word) {
+                                          int* err_word, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t polls = 0;
@@ -75,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (mbar_try_wait(bar, parity)) return true;
     if ((++polls & 255u) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicOr(err_word, 1);
         return false;

@@ -110,9 +110,17 @@ extern "C" int cascade_accept_static(int32_t B, int32_t T, const int32_t* parent
   for (int j = 0; j < T; ++j)
     for (int i = j; i >= 0; i = h_parent[i]) anc[(size_t)j * 4 + (i >> 6)] |= 1ull << (i & 63);
 
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The copies below read host memory that lives only until this call returns: a stream that is recording
+  // would replay them later from memory that is gone, so it is refused.
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return CASCADE_ERR_CUDA;
+  }
+  if (capturing != cudaStreamCaptureStatusNone) return CASCADE_ERR_INVALID_ARG;
   unsigned char* base = nullptr;
   CASCADE_TRY(scratch_address(&base));
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   // The array still holds the previous call's descriptor and scores: everything read below is rewritten
   // here, and the counters (which the kernel expects at zero) are cleared.
   CASCADE_CUDA_TRY(cudaMemcpyAsync(base + Layout::off_ints, ints.data(), Layout::kInts * 4, cudaMemcpyHostToDevice, s));

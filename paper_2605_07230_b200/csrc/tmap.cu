@@ -4,7 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <cstring>
-#include <deque>
+#include <list>
 #include <vector>
 
 #include "cascade_internal.h"
@@ -25,8 +25,12 @@ struct Entry {
   alignas(64) CUtensorMap map;
 };
 
+// Least recently used first.  A list never moves its elements, so a pointer to a map stays valid until that
+// entry is evicted -- and only the entry that has gone unused for longest ever is, thousands of lookups after
+// its last use, never one that the call in progress (a dozen maps at most) has fetched.
+constexpr size_t kMaxEntries = 4096;
 struct Cache {
-  std::deque<Entry> entries;  // deque: growth never moves existing maps
+  std::list<Entry> entries;
 };
 
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
@@ -44,11 +48,14 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 const CUtensorMap* lookup_or_make(cascade_ctx* ctx, const Key& key) {
   if (ctx->tmap_cache == nullptr) ctx->tmap_cache = new Cache();
   Cache* c = static_cast<Cache*>(ctx->tmap_cache);
-  for (const Entry& e : c->entries)
-    if (e.key == key) return &e.map;
+  for (auto it = c->entries.begin(); it != c->entries.end(); ++it)
+    if (it->key == key) {
+      c->entries.splice(c->entries.end(), c->entries, it);  // most recently used last; the element stays where it is in memory
+      return &it->map;
+    }
   auto fn = encode_fn();
   if (fn == nullptr) return nullptr;
-  if (c->entries.size() > 4096) c->entries.clear();  // unbounded pointer churn: start over
+  if (c->entries.size() >= kMaxEntries) c->entries.pop_front();  // callers that churn through buffers
   c->entries.emplace_back();
   Entry& e = c->entries.back();
   std::memset(&e.key, 0, sizeof(Key));

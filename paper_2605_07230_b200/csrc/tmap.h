@@ -7,7 +7,8 @@ struct cascade_ctx;
 
 // Tiled map over a row-major bf16 matrix [rows][cols] (cols contiguous) with a box of
 // [box_rows][box_cols]; box_cols * 2 bytes must be <= 128 and is the 128-byte-swizzle span.
-// Returns nullptr on failure.  The returned pointer stays valid for the life of the context.
+// Returns nullptr on failure.  The returned pointer stays valid at least until 4000 other maps have been
+// looked up on the context (the cache evicts the map that has gone unused for longest).
 const CUtensorMap* get_tmap_2d_bf16(cascade_ctx* ctx, const void* base, uint64_t rows, uint64_t cols,
                                     uint64_t row_stride_elems, uint32_t box_rows, uint32_t box_cols);
 

@@ -226,14 +226,16 @@ class DecodeLoop:
     argument marshalling only."""
 
     def __init__(self, w: synth.Workload, n_layers: int, max_steps: int, device="cuda:0", seed: int = 0,
-                 select_mode: int = cb.SELECT_LONGEST, tile_layers: bool = False):
+                 select_mode: int = cb.SELECT_LONGEST, tile_layers: bool = False, cap: int | None = None):
         # tile_layers: every layer gets the values of one seeded layer (its own copy on the device, its own
         # caches): for timing at full depth without generating 30 layers of weights on the host
         self.w, self.n_layers, self.device = w, n_layers, device
         self.parent = w.parent()
         T = self.T = len(self.parent)
         depth = int(synth.tree_depth(self.parent).max())
-        self.cap = w.prefix_len + max_steps * (depth + 1)
+        # rows per cache: room for `max_steps` steps that each accept a whole path, unless the caller knows better
+        # (a run that stops at a token count); a step that does not fit is refused by the library, not written
+        self.cap = cap if cap is not None else w.prefix_len + max_steps * (depth + 1)
         B, R = w.B, 2 * w.B
         self.ctx = cb.Context(cb.BF16 if w.dtype == "bf16" else cb.F32, B, T, self.cap, w.h, w.n_heads, w.n_heads,
                               w.head_dim, w.V, w.ffn)

@@ -1,0 +1,86 @@
+"""GPU parity at the sizes the benchmark runs: the Janus-Pro-7B- and Lumina-mGPT-7B-768-shaped verification
+steps through one full-width decoder layer (hidden 4096, 32 heads x 128, SwiGLU 11008, vocabulary 16384 / 65536,
+prefix 384 / 2480, 61 tree rows), the LM head alone at vocabulary 65536 with 61 and 122 rows, and the tree
+attention alone at 32 heads over a 2480-key prefix -- every output element against the fp64 checker on the same
+seeded inputs.  These are the launch configurations bench.py times: the projections' sliced and balanced modes with
+dozens of units per CTA, the head's contiguous mode with several whole tiles per CTA and both hand-off roles in
+one CTA, the attention with 32 heads x 2 splits."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cascade_oracle as O
+from paper_2605_07230_b200 import binding as cb
+from paper_2605_07230_b200 import synth
+from paper_2605_07230_b200.workload import LayerWorkload
+from tests import gpu_util as G
+from tests.test_gpu_attention import ATTN_TOL, run_attention
+from tests.test_gpu_head import LOGIT_TOL, run_head
+
+pytestmark = pytest.mark.gpu
+
+HIDDEN_TOL = 2e-2
+
+
+@pytest.mark.parametrize("name", ["janus", "lumina"])
+def test_full_width_step_through_one_layer(name):
+    w = synth.workload(name)
+    wl = LayerWorkload(w, n_layers=1, keep_logits=True)
+    s = wl.run(0)
+    torch.cuda.synchronize()
+    wl.ctx.check()
+    h = s.host
+    ref = O.verify_step(h["embed"], h["layers"], h["gamma_final"], h["w_head"], h["tok"], wl.parent, h["k_prefix"],
+                        h["v_prefix"], h["prefix_len"], h["draft_p"], h["uniforms"], w.n_heads, w.head_dim, w.eps,
+                        w.rope_base, w.cfg_scale, 1.0, w.tau_pos, w.tau_seq, w.tvd_budget, kv_bf16=True)
+    q, k, v = ref["attn_io"][0]
+    k_err = np.abs(s.out["k_tree_out"][0].float().cpu().numpy() - k).max()
+    v_err = np.abs(s.out["v_tree_out"][0].float().cpu().numpy() - v).max()
+    assert k_err < 4e-2 and v_err < 4e-2, (k_err, v_err)       # one bf16 step at |k| up to ~8
+    hid_err = np.abs(s.out["hidden_out"].cpu().numpy() - ref["hidden"]).max()
+    assert hid_err < HIDDEN_TOL, hid_err
+    logits = s.out["logits"].cpu().numpy()
+    logit_err = np.abs(logits - ref["head"]["logits"]).max()
+    assert logit_err < LOGIT_TOL, logit_err
+    assert np.abs(s.out["row_lse"].cpu().numpy() - ref["head"]["lse"]).max() < 3e-3
+    assert np.abs(s.out["feat"].cpu().numpy() - ref["head"]["feat"]).max() < 2e-2
+    # decisions: the checker's rule on the device's own features and logits, bit-exact outside the near band
+    feat = s.out["feat"].cpu().numpy().astype(np.float64)
+    rows = [O.relaxed_accept(feat[b], logits[b], h["tok"][b], wl.parent, h["draft_p"][b], h["uniforms"][b], w.tau_pos,
+                             w.tau_seq, w.tvd_budget) for b in range(w.B)]
+    st = G.compare_decisions(wl.parent, rows, s.out["accept"].cpu().numpy(), s.out["path_nodes"].cpu().numpy(),
+                             s.out["path_len"].cpu().numpy(), cb.SELECT_LONGEST)
+    # the checker end to end (its own hidden states and logits): reported, with a loose floor
+    agree = float(np.mean([np.mean(s.out["accept"][b].cpu().numpy() == ref["accept"][b]["accept"]) for b in range(w.B)]))
+    assert agree >= 0.9, agree
+    print(f"{name} full width: k/v {k_err:.1e}/{v_err:.1e}, hidden {hid_err:.2e}, logits {logit_err:.2e}, "
+          f"{wl.ctx.last_launch_count} kernels, nodes compared {st['nodes_compared']}/{st['nodes']}, set aside "
+          f"{st['nodes_set_aside']}, device near count {s.out['near_count'].cpu().tolist()}, end-to-end node agreement "
+          f"{agree:.3f}, path lengths {s.out['path_len'].cpu().tolist()}")
+    wl.close()
+
+
+@pytest.mark.parametrize("B", [1, 2])
+def test_head_at_vocabulary_65536(B):
+    """61 and 122 activation rows against a [65536, 4096] head: 512 vocabulary tiles x 32 K blocks over 148 CTAs, so
+    every CTA holds whole tiles, finishes a tile another CTA began and hands its last one on."""
+    w = synth.workload("lumina", B=B)
+    parent = w.parent()
+    got, ref, tok = run_head(w, parent, 41)
+    err = np.abs(got["logits"] - ref["logits"]).max()
+    assert err < LOGIT_TOL, err
+    assert np.abs(got["feat"] - ref["feat"]).max() < 1e-4
+    assert np.abs(got["lse"] - ref["lse"]).max() < 2e-3
+    lp, lg = O.candidate_logits(ref["logits"], tok, parent)
+    assert np.abs(got["cp"] - lp).max() < 2e-3 and np.abs(got["cg"] - lg).max() < 2e-3
+    print(f"head V=65536, {B * len(parent)} rows: logits max-abs {err:.2e}")
+
+
+@pytest.mark.parametrize("name", ["janus", "lumina"])
+def test_attention_at_32_heads(name):
+    w = synth.workload(name)
+    got, ref, _ = run_attention(w, w.parent(), 43)
+    assert np.isfinite(got).all()
+    err = np.abs(got - ref).max()
+    assert err < ATTN_TOL, err
+    print(f"attention {name}: 32 heads, prefix {w.prefix_len}, max-abs {err:.2e}")

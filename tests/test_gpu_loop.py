@@ -15,13 +15,16 @@ from tests import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("over,n_layers,steps,graph_after", [
-    (dict(B=2, tree="topk32", prefix_len=40), 2, 3, None),
-    (dict(B=1, tree="topk60", prefix_len=130), 3, 2, None),
-    (dict(B=2, tree="topk32", prefix_len=40), 2, 4, 1),     # steps after the first replay a recorded CUDA graph
+@pytest.mark.parametrize("name,over,n_layers,steps,graph_after", [
+    ("mini", dict(B=2, tree="topk32", prefix_len=40), 2, 3, None),
+    ("mini", dict(B=1, tree="topk60", prefix_len=130), 3, 2, None),
+    ("mini", dict(B=2, tree="topk32", prefix_len=40), 2, 4, 1),     # steps after the first replay a recorded CUDA graph
+    # the decode loop's own widths (hidden 4096, 32 heads x 128, SwiGLU 11008, vocabulary 16384, 64-row prompt cache,
+    # 61-row trees): two of its layers, two steps, the second replayed from a recorded graph
+    ("janus", dict(prefix_len=64), 2, 2, 1),
 ])
-def test_decode_loop(over, n_layers, steps, graph_after):
-    w = synth.workload("mini", **over)
+def test_decode_loop(name, over, n_layers, steps, graph_after):
+    w = synth.workload(name, **over)
     loop = DecodeLoop(w, n_layers, max_steps=steps, seed=11)
     B, parent = w.B, loop.parent
     h = loop.host
