@@ -19,9 +19,6 @@ pytestmark = pytest.mark.gpu
     ("mini", dict(B=2, tree="topk32", prefix_len=40), 2, 3, None),
     ("mini", dict(B=1, tree="topk60", prefix_len=130), 3, 2, None),
     ("mini", dict(B=2, tree="topk32", prefix_len=40), 2, 4, 1),     # steps after the first replay a recorded CUDA graph
-    # the decode loop's own widths (hidden 4096, 32 heads x 128, SwiGLU 11008, vocabulary 16384, 64-row prompt cache,
-    # 61-row trees): two of its layers, two steps, the second replayed from a recorded graph
-    ("janus", dict(prefix_len=64), 2, 2, 1),
 ])
 def test_decode_loop(name, over, n_layers, steps, graph_after):
     w = synth.workload(name, **over)
