@@ -37,7 +37,8 @@ extern "C" {
 /* ---- status codes ------------------------------------------------------------------------------ */
 #define CASCADE_OK 0
 #define CASCADE_ERR_INVALID_ARG (-1)       /* null pointer, non-positive size, value out of range     */
-#define CASCADE_ERR_BAD_TREE (-2)          /* parent[] is not a BFS-ordered tree with grouped siblings */
+#define CASCADE_ERR_BAD_TREE (-2)          /* parent[] is not a BFS-ordered tree with grouped siblings (from
+                                              cascade_check: found by cascade_tree_update_device)        */
 #define CASCADE_ERR_WORKSPACE (-3)         /* device allocation of the context's scratch failed        */
 #define CASCADE_ERR_UNSUPPORTED_SHAPE (-4) /* shape outside what the kernels handle (see cascade_shape) */
 #define CASCADE_ERR_CUDA (-5)              /* a CUDA runtime / driver call failed                      */
@@ -101,8 +102,8 @@ int cascade_destroy(cascade_ctx* ctx);
 int64_t cascade_workspace_bytes(const cascade_ctx* ctx);
 
 /* Reads the context's device-side error word (set when a bounded wait inside a kernel ran out) after
- * synchronising `stream`.  Returns CASCADE_OK, CASCADE_ERR_TIMEOUT, CASCADE_ERR_OVERFLOW or CASCADE_ERR_CUDA, and clears
- * the word. */
+ * synchronising `stream`.  Returns CASCADE_OK, CASCADE_ERR_TIMEOUT, CASCADE_ERR_BAD_TREE, CASCADE_ERR_OVERFLOW or
+ * CASCADE_ERR_CUDA, and clears the word. */
 int cascade_check(cascade_ctx* ctx, void* stream);
 
 /* Number of kernels the most recent call on this context enqueued. */
@@ -148,6 +149,27 @@ int cascade_tree_destroy(cascade_tree* tree);
  * An invalid tree returns its error and leaves the descriptor as it was.  Host-side queries
  * (cascade_tree_rows / depth / num_pairs / pairs) answer for the new tree as soon as the call returns. */
 int cascade_tree_update(cascade_tree* tree, int32_t T, const int32_t* parent, void* stream);
+/* The same, from a parent[] that is already in DEVICE memory, without a host round trip (drafters that decide
+ * the tree's shape on the device each step: the dynamic trees that Section 2 contrasts with the static mask).
+ * One small kernel on `stream` checks the rules of cascade_tree_create and writes the descriptor.  The host
+ * cannot see the tree, so the caller states bounds that sizes depend on:
+ *   T          rows (host value; grids and row counts of every later call come from it), <= T_max;
+ *   depth_cap  the tree is at most this deep; path_nodes arrays of later calls have depth_cap + 1 entries per
+ *              prompt and cascade_tree_depth returns it;
+ *   pairs_cap  at most this many (node, node) pairs (edges + sibling pairs); scores arrays of later calls have
+ *              pairs_cap entries per prompt and cascade_tree_num_pairs returns it; <= 0: the context's maximum.
+ * A parent[] that breaks a rule or a bound is found on the device: cascade_check then returns
+ * CASCADE_ERR_BAD_TREE, and the descriptor is left holding a neutral tree of T rows (every row a childless leaf
+ * below the root, no pairs), so that calls already enqueued behind it stay within their buffers; their results
+ * are meaningless.  Nothing is allocated; the host-side mirrors are not refreshed (cascade_tree_pairs and
+ * cascade_tree_download fetch from the device with blocking copies). */
+int cascade_tree_update_device(cascade_tree* tree, int32_t T, int32_t depth_cap, int32_t pairs_cap,
+                               const int32_t* parent_dev, void* stream);
+/* Copies the descriptor's device arrays to HOST arrays (blocking copies; synchronise the stream of a pending
+ * update first): parent, depth, child_begin, child_count [T] int32 and the packed ancestor-or-self mask
+ * anc [T][4] uint64 (bit i of row j set iff i is j or an ancestor of j).  Any pointer may be NULL. */
+int cascade_tree_download(const cascade_tree* tree, int32_t* parent, int32_t* depth, int32_t* child_begin,
+                          int32_t* child_count, uint64_t* anc);
 int32_t cascade_tree_rows(const cascade_tree* tree);      /* T                                     */
 int32_t cascade_tree_depth(const cascade_tree* tree);     /* deepest level                         */
 int32_t cascade_tree_num_pairs(const cascade_tree* tree); /* edges + sibling pairs                 */
@@ -326,18 +348,23 @@ int cascade_verify_step_host(cascade_ctx* ctx, const cascade_tree* tree, const c
                              void* stream);
 
 /* ---- between two steps of a decode loop --------------------------------------------------------- */
-/* The token after the accepted path: Algorithm 1's last step (the next token is drawn from the target
- * distribution with the rejected proposals removed; from the target distribution itself after a fully
- * accepted draft), which Algorithm 2 leaves out.  For prompt b, end = last node of its path; the tokens of
- * end's children (all rejected, whichever selection mode chose the path) get probability zero, the rest of
- * softmax(logits[b, end, :]) is renormalised, and token_out[b] is the inverse-CDF sample at u_bonus[b]:
- * the first v whose cumulative weight exceeds u_bonus[b] * (remaining weight).
+/* The token after the accepted path: Algorithm 1's last step, which Algorithm 2 leaves out.  For prompt b,
+ * end = last node of its path, q = softmax(logits[b, end, :]).  Two rules:
+ *   draft_row != NULL (the drafter's full distribution p at the end node, [B,V] float, row b for prompt b):
+ *     Algorithm 1's correction step -- if a child of end was rejected, the token is drawn from [q - p]+
+ *     normalised; after a fully accepted draft (end has no children), from q.  Should nothing of q lie above p
+ *     (p = q), q is used.  mass_out[b] = sum of [q - p]+ (1 where q was used).
+ *   draft_row == NULL (a tree drafter that keeps only the probabilities of its proposals): the tokens of end's
+ *     children (all rejected, whichever selection mode chose the path) get probability zero, the rest of q is
+ *     renormalised.  mass_out[b] = the probability mass that remains.
+ * token_out[b] is the inverse-CDF sample at u_bonus[b]: the first v whose cumulative weight exceeds
+ * u_bonus[b] * (total weight).
  *   logits [B,T,V] float (as stored by cascade_lm_head_cfg / cascade_verify_step); tok [B,T] int32;
  *   path_nodes [B,depth+1], path_len [B] from cascade_select_path; u_bonus [B] float in [0,1);
- *   token_out [B] int32; mass_out [B] float or NULL: remaining probability mass after the removal. */
+ *   token_out [B] int32; mass_out [B] float or NULL. */
 int cascade_bonus_token(cascade_ctx* ctx, const cascade_tree* tree, const float* logits, const int32_t* tok,
-                        const int32_t* path_nodes, const int32_t* path_len, const float* u_bonus, int32_t* token_out,
-                        float* mass_out, void* stream);
+                        const float* draft_row, const int32_t* path_nodes, const int32_t* path_len,
+                        const float* u_bonus, int32_t* token_out, float* mass_out, void* stream);
 
 /* Appends the keys / values of the accepted path's tree rows (root row first: the pending token, then the
  * accepted drafts) to the caches of n_layers layers, for both CFG rows of every prompt, at positions

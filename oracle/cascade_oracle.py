@@ -17,6 +17,7 @@ Parity pins (tests/test_oracle_*.py): every function below is pinned to somethin
 textbook causal / decode attention, CFG end points and linearity, closed-form cosine cases, reduction
 to Algorithm 1 with the relaxation off, an independently written sequential walk of Algorithm 2,
 brute-force path enumeration, threshold monotonicity with an unbounded budget, hand-computed trees,
+exact recovery of the target distribution by accept test + residual draw (Algorithm 1's guarantee),
 the library's top-k and a brute-force nucleus for the truncation of the target distribution.
 `decoder_layer` (architecture from the workload definition, not from the paper) is pinned against an
 ordinary causal block built from torch's library routines: on a chain with an empty prefix, and on a
@@ -377,6 +378,25 @@ def bonus_token(logits_row, rejected_tokens, u):
     c = np.cumsum(g)
     v = int(np.searchsorted(c, float(u) * total, side="right"))
     return min(v, len(g) - 1), total
+
+
+def residual_token(logits_row, draft_row, any_rejected, u):
+    """Algorithm 1's last step, literally: after a rejection the next token is drawn from the positive part of
+    (target - drafter), renormalised,  [q - p]+ / sum [q - p]+ , with q = softmax(logits_row) and p the drafter's
+    distribution at the same position; after a fully accepted draft (nothing rejected) it is drawn from q.  The
+    draw is the inverse-CDF sample at u in [0,1): the first v with cumsum(weight)[v] > u * total.  Where nothing of
+    q lies above p (p = q; Algorithm 1 then never rejects) q itself is used.  Returns (token, total), total = the
+    sum of [q - p]+ (1.0 where q was used)."""
+    q = softmax(np.asarray(logits_row, np.float64))
+    w = q
+    total = 1.0
+    if any_rejected:
+        r = np.maximum(q - np.asarray(draft_row, np.float64), 0.0)
+        if r.sum() > 0.0:
+            w, total = r, float(r.sum())
+    c = np.cumsum(w)
+    v = int(np.searchsorted(c, float(u) * c[-1], side="right"))
+    return min(v, len(w) - 1), total
 
 
 def filter_logits(logits, top_k, top_p):

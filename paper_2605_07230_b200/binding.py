@@ -30,6 +30,7 @@ EXPORTS = [
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
     "cascade_verify_step_host", "cascade_accept_static", "cascade_bonus_token", "cascade_kv_append",
     "cascade_filter_logits", "cascade_set_wait_limit", "cascade_wait_probe",
+    "cascade_tree_update_device", "cascade_tree_download",
 ]
 
 
@@ -103,9 +104,11 @@ def lib() -> C.CDLL:
         L.cascade_verify_step_host.argtypes = [vp, vp, C.POINTER(Step), vp, vp, vp, vp, vp, vp, vp]
         L.cascade_accept_static.argtypes = [C.c_int32, C.c_int32, vp, vp, C.c_int32, vp, vp, vp, vp, vp, vp, vp,
                                             C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp, vp]
-        L.cascade_bonus_token.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.cascade_bonus_token.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.cascade_kv_append.argtypes = [vp, vp, C.c_int32, C.POINTER(Layer), vp, vp, vp, vp, C.c_int32, vp, vp]
         L.cascade_filter_logits.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_float, vp, vp]
+        L.cascade_tree_update_device.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, vp, vp]
+        L.cascade_tree_download.argtypes = [vp, vp, vp, vp, vp, vp]
         L.cascade_set_wait_limit.argtypes = [vp, C.c_int64]
         L.cascade_wait_probe.argtypes = [vp, vp, vp]
         _lib = L
@@ -210,6 +213,21 @@ class Tree:
         self.T = lib().cascade_tree_rows(self.handle)
         self.depth = lib().cascade_tree_depth(self.handle)
         self.num_pairs = lib().cascade_tree_num_pairs(self.handle)
+
+    def update_device(self, T: int, depth_cap: int, pairs_cap: int, parent_dev):
+        """A new tree from a device-resident int32 parent[] (no host round trip); enqueued on the current stream."""
+        _check(lib().cascade_tree_update_device(self.handle, T, depth_cap, pairs_cap, _ptr(parent_dev), _stream()))
+        self.T = lib().cascade_tree_rows(self.handle)
+        self.depth = lib().cascade_tree_depth(self.handle)
+        self.num_pairs = lib().cascade_tree_num_pairs(self.handle)
+
+    def download(self):
+        """The descriptor's device arrays as host lists: parent, depth, child_begin, child_count, anc (T x 4 words)."""
+        T = self.T
+        arrs = [(C.c_int32 * T)() for _ in range(4)]
+        anc = (C.c_uint64 * (4 * T))()
+        _check(lib().cascade_tree_download(self.handle, *arrs, anc))
+        return [list(a) for a in arrs] + [[list(anc[4 * j: 4 * j + 4]) for j in range(T)]]
 
     def pairs(self):
         a = (C.c_int32 * max(self.num_pairs, 1))()
@@ -324,9 +342,11 @@ def cascade_filter_logits(ctx, logits, top_k, top_p, kept_count=None):
                                        _stream()))
 
 
-def cascade_bonus_token(ctx, tree, logits, tok, path_nodes, path_len, u_bonus, token_out, mass_out=None):
-    _check(lib().cascade_bonus_token(ctx.handle, tree.handle, _ptr(logits), _ptr(tok), _ptr(path_nodes),
-                                     _ptr(path_len), _ptr(u_bonus), _ptr(token_out), _ptr(mass_out), _stream()))
+def cascade_bonus_token(ctx, tree, logits, tok, path_nodes, path_len, u_bonus, token_out, mass_out=None,
+                        draft_row=None):
+    _check(lib().cascade_bonus_token(ctx.handle, tree.handle, _ptr(logits), _ptr(tok), _ptr(draft_row),
+                                     _ptr(path_nodes), _ptr(path_len), _ptr(u_bonus), _ptr(token_out),
+                                     _ptr(mass_out), _stream()))
 
 
 def cascade_kv_append(ctx, tree, step: Step, k_tree, v_tree, path_nodes, path_len, prefix_cap, prefix_len):

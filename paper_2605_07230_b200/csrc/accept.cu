@@ -42,9 +42,12 @@ __device__ __forceinline__ float warp_max(float v) {
 
 struct TreeDev {
   int T, depth_max, n_pairs;
+  int pairs_stride;     // row length of the scores arrays (= n_pairs unless the tree was built on the device)
+  const int32_t* meta;  // device-built tree: meta[0] = its pair count (the host does not know it); else null
   const int32_t *parent, *depth, *child_begin, *child_count, *sib_base, *pair_a, *pair_b;
   const uint64_t* anc;
 };
+__device__ __forceinline__ int pair_count(const TreeDev& tr) { return tr.meta != nullptr ? tr.meta[0] : tr.n_pairs; }
 
 struct AcceptIO {
   const float* scores;        // [B, n_pairs]
@@ -71,6 +74,7 @@ struct TailArgs {
   int feat_dim;
   const float* feat_norm;
   float* scores_out;
+  int n_pair_blocks;  // CTAs per prompt that take cosines (each strides over the pair list)
   // row log-sum-exp from the LM head's partials
   const float2* part;
   int part_ld, n_tiles, n_lse_blocks;
@@ -99,7 +103,8 @@ __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
   const int T = tr.T, j = threadIdx.x;
   const size_t row0 = (size_t)b * T;
   const cascade_params prm = io.prm;
-  for (int i = j; i < tr.n_pairs; i += kTailThreads) s_scores[i] = __ldcg(io.scores + (size_t)b * tr.n_pairs + i);
+  const int n_pairs = min(pair_count(tr), tr.pairs_stride);
+  for (int i = j; i < n_pairs; i += kTailThreads) s_scores[i] = __ldcg(io.scores + (size_t)b * tr.pairs_stride + i);
   // every global read of this block is issued here, in one round trip
   float my_p = 0.f, my_u = 1.f, my_cp = 0.f, my_cg = 0.f;
   uint64_t my_anc[kMaxT / 64] = {0, 0, 0, 0};
@@ -300,45 +305,49 @@ __device__ void accept_block(const TreeDev& tr, const AcceptIO& io, int b) {
 __global__ void __launch_bounds__(kTailThreads) k_tail(const TreeDev tr, const TailArgs ta, const AcceptIO io) {
   const int b = blockIdx.y, blk = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_pair_blocks = ta.feat != nullptr ? tr.n_pairs : 0;
+  const int n_pair_blocks = ta.feat != nullptr ? ta.n_pair_blocks : 0;
   if (blk < n_pair_blocks) {
-    // cosine of one pair
+    // cosines: one pair per CTA when the host knows the pair count, a strided share of the list otherwise
     __shared__ float red[3][kTailThreads / 32];
-    const int ia = tr.pair_a[blk], ib = tr.pair_b[blk];
-    const float4* fa = reinterpret_cast<const float4*>(ta.feat + ((size_t)b * tr.T + ia) * ta.feat_dim);
-    const float4* fb = reinterpret_cast<const float4*>(ta.feat + ((size_t)b * tr.T + ib) * ta.feat_dim);
-    float dot = 0.f, na = 0.f, nb = 0.f;
-    for (int i = threadIdx.x; i < ta.feat_dim / 4; i += kTailThreads) {
-      const float4 x = fa[i], y = fb[i];
-      dot += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
-      na += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-      nb += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
-    }
-    dot = warp_sum(dot);
-    na = warp_sum(na);
-    nb = warp_sum(nb);
-    if (lane == 0) {
-      red[0][warp] = dot;
-      red[1][warp] = na;
-      red[2][warp] = nb;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      dot = na = nb = 0.f;
-      for (int w = 0; w < kTailThreads / 32; ++w) {
-        dot += red[0][w];
-        na += red[1][w];
-        nb += red[2][w];
+    const int n_pairs = min(pair_count(tr), tr.pairs_stride);
+    for (int pi = blk; pi < n_pairs; pi += n_pair_blocks) {
+      const int ia = tr.pair_a[pi], ib = tr.pair_b[pi];
+      const float4* fa = reinterpret_cast<const float4*>(ta.feat + ((size_t)b * tr.T + ia) * ta.feat_dim);
+      const float4* fb = reinterpret_cast<const float4*>(ta.feat + ((size_t)b * tr.T + ib) * ta.feat_dim);
+      float dot = 0.f, na = 0.f, nb = 0.f;
+      for (int i = threadIdx.x; i < ta.feat_dim / 4; i += kTailThreads) {
+        const float4 x = fa[i], y = fb[i];
+        dot += x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
+        na += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+        nb += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
       }
-      float norm_a, norm_b;
-      if (ta.feat_norm != nullptr) {
-        norm_a = ta.feat_norm[(size_t)b * tr.T + ia];
-        norm_b = ta.feat_norm[(size_t)b * tr.T + ib];
-      } else {
-        norm_a = sqrtf(na);
-        norm_b = sqrtf(nb);
+      dot = warp_sum(dot);
+      na = warp_sum(na);
+      nb = warp_sum(nb);
+      __syncthreads();  // the previous pair's sums have been read
+      if (lane == 0) {
+        red[0][warp] = dot;
+        red[1][warp] = na;
+        red[2][warp] = nb;
       }
-      ta.scores_out[(size_t)b * tr.n_pairs + blk] = dot / (norm_a * norm_b);
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        dot = na = nb = 0.f;
+        for (int w = 0; w < kTailThreads / 32; ++w) {
+          dot += red[0][w];
+          na += red[1][w];
+          nb += red[2][w];
+        }
+        float norm_a, norm_b;
+        if (ta.feat_norm != nullptr) {
+          norm_a = ta.feat_norm[(size_t)b * tr.T + ia];
+          norm_b = ta.feat_norm[(size_t)b * tr.T + ib];
+        } else {
+          norm_a = sqrtf(na);
+          norm_b = sqrtf(nb);
+        }
+        ta.scores_out[(size_t)b * tr.pairs_stride + pi] = dot / (norm_a * norm_b);
+      }
     }
   } else if (blk < n_pair_blocks + ta.n_lse_blocks) {
     // log-sum-exp of one logits row per warp from the per-tile (max, sum of exp) partials
@@ -515,6 +524,8 @@ TreeDev tree_dev(const cascade_tree* tree) {
   t.T = tree->T;
   t.depth_max = tree->depth_max;
   t.n_pairs = tree->n_pairs;
+  t.pairs_stride = tree->n_pairs;
+  t.meta = tree->device_built ? tree->d_meta : nullptr;
   t.parent = tree->d_parent;
   t.depth = tree->d_depth;
   t.child_begin = tree->d_child_begin;
@@ -537,6 +548,9 @@ int launch_tail(cascade_ctx* ctx, const cascade_tree* tree, const TailWork& w, c
     ta.feat_dim = w.feat_dim;
     ta.feat_norm = w.feat_norm;
     ta.scores_out = w.scores;
+    // a tree built on the device has an unknown number of pairs (n_pairs is then the row length it may fill):
+    // a fixed number of CTAs shares the list
+    ta.n_pair_blocks = tree->device_built ? (tree->n_pairs < 128 ? tree->n_pairs : 128) : tree->n_pairs;
   }
   if (w.part != nullptr) {
     ta.part = w.part;
@@ -565,7 +579,7 @@ int launch_tail(cascade_ctx* ctx, const cascade_tree* tree, const TailWork& w, c
     io.path_len = w.path_len;
     io.tvd_used = w.tvd_used;
   }
-  int blocks = (ta.feat != nullptr ? tree->n_pairs : 0) + ta.n_lse_blocks;
+  int blocks = (ta.feat != nullptr ? ta.n_pair_blocks : 0) + ta.n_lse_blocks;
   if (blocks == 0) {
     if (!ta.do_accept) return CASCADE_OK;
     blocks = 1;  // nothing to prepare: a single CTA per prompt runs the rule

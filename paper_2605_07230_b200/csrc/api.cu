@@ -157,7 +157,7 @@ const char* cascade_kernel_name(int32_t id) {
   static const char* names[] = {"tree_attn", "tree_attn_f32", "final_norm_mix", "gemm_head",
                                 "head_f32", "row_stats", "row_lse", "similarity", "accept", "tail", "select_path",
                                 "embed_norm", "gemm_qkv", "rope_split", "gemm_o", "resid_norm", "gemm_gate_up",
-                                "swiglu", "gemm_down", "gemm_f32", "resid_add", "kv_append", "bonus_token", "filter_logits", "wait_probe"};
+                                "swiglu", "gemm_down", "gemm_f32", "resid_add", "kv_append", "bonus_token", "filter_logits", "wait_probe", "build_tree"};
   static_assert(sizeof(names) / sizeof(names[0]) == K_KERNEL_ID_END, "one name per kernel id");
   if (id < 0 || id >= K_KERNEL_ID_END) return nullptr;
   return names[id];
@@ -262,7 +262,8 @@ int cascade_check(cascade_ctx* ctx, void* stream) {
   if (word != 0) {
     CASCADE_CUDA_TRY(cudaMemsetAsync(ctx->dev_error, 0, sizeof(int), s));
     CASCADE_CUDA_TRY(cudaStreamSynchronize(s));
-    return (word & CASCADE_DEV_ERR_WAIT) ? CASCADE_ERR_TIMEOUT : CASCADE_ERR_OVERFLOW;
+    if (word & CASCADE_DEV_ERR_WAIT) return CASCADE_ERR_TIMEOUT;
+    return (word & CASCADE_DEV_ERR_BAD_TREE) ? CASCADE_ERR_BAD_TREE : CASCADE_ERR_OVERFLOW;
   }
   return CASCADE_OK;
 }
@@ -345,6 +346,7 @@ int install_host_tree(cascade_tree* t, HostTree&& h, cudaStream_t s, bool async)
   t->depth_max = h.depth_max;
   t->n_pairs = h.n_pairs;
   t->uid = next_tree_uid();
+  t->device_built = false;
   t->parent = std::move(h.parent);
   t->depth = std::move(h.depth);
   t->child_begin = std::move(h.child_begin);
@@ -377,6 +379,7 @@ int cascade_tree_create(cascade_ctx* ctx, int32_t T, const int32_t* parent, casc
     cv.take(t->d_pair_a, pairs_cap);
     cv.take(t->d_pair_b, pairs_cap);
     cv.take(t->d_anc, T_cap * 4);
+    cv.take(t->d_meta, 4);
     return align_up(cv.off, 256);
   };
   const int64_t bytes = layout(nullptr);
@@ -403,6 +406,24 @@ int cascade_tree_update(cascade_tree* tree, int32_t T, const int32_t* parent, vo
   return install_host_tree(tree, std::move(h), as_stream(stream), true);
 }
 
+int cascade_tree_update_device(cascade_tree* tree, int32_t T, int32_t depth_cap, int32_t pairs_cap,
+                               const int32_t* parent_dev, void* stream) {
+  if (tree == nullptr || parent_dev == nullptr || T < 1 || depth_cap < 0) return CASCADE_ERR_INVALID_ARG;
+  cascade_ctx* ctx = tree->ctx;
+  if (T > ctx->shape.T_max) return CASCADE_ERR_UNSUPPORTED_SHAPE;
+  if (T > 1 && depth_cap < 1) return CASCADE_ERR_INVALID_ARG;
+  if (depth_cap > T - 1) depth_cap = T - 1;
+  if (pairs_cap <= 0 || pairs_cap > ctx->max_pairs) pairs_cap = ctx->max_pairs;
+  ctx->launches = 0;
+  CASCADE_TRY(launch_build_tree(ctx, tree, T, depth_cap, pairs_cap, parent_dev, as_stream(stream)));
+  tree->T = T;
+  tree->depth_max = depth_cap;
+  tree->n_pairs = pairs_cap;
+  tree->device_built = true;
+  tree->uid = next_tree_uid();
+  return CASCADE_OK;
+}
+
 int cascade_tree_destroy(cascade_tree* tree) {
   if (tree == nullptr) return CASCADE_ERR_INVALID_ARG;
   // steps recorded by the host-buffer entry point into this descriptor's device arrays
@@ -419,11 +440,35 @@ int cascade_tree_destroy(cascade_tree* tree) {
   return CASCADE_OK;
 }
 
+int cascade_tree_download(const cascade_tree* tree, int32_t* parent, int32_t* depth, int32_t* child_begin,
+                          int32_t* child_count, uint64_t* anc) {
+  if (tree == nullptr) return CASCADE_ERR_INVALID_ARG;
+  const size_t n = sizeof(int32_t) * (size_t)tree->T;
+  if (parent != nullptr) CASCADE_CUDA_TRY(cudaMemcpy(parent, tree->d_parent, n, cudaMemcpyDeviceToHost));
+  if (depth != nullptr) CASCADE_CUDA_TRY(cudaMemcpy(depth, tree->d_depth, n, cudaMemcpyDeviceToHost));
+  if (child_begin != nullptr) CASCADE_CUDA_TRY(cudaMemcpy(child_begin, tree->d_child_begin, n, cudaMemcpyDeviceToHost));
+  if (child_count != nullptr) CASCADE_CUDA_TRY(cudaMemcpy(child_count, tree->d_child_count, n, cudaMemcpyDeviceToHost));
+  if (anc != nullptr)
+    CASCADE_CUDA_TRY(cudaMemcpy(anc, tree->d_anc, sizeof(uint64_t) * 4 * (size_t)tree->T, cudaMemcpyDeviceToHost));
+  return CASCADE_OK;
+}
+
 int32_t cascade_tree_rows(const cascade_tree* tree) { return tree ? tree->T : 0; }
 int32_t cascade_tree_depth(const cascade_tree* tree) { return tree ? tree->depth_max : 0; }
 int32_t cascade_tree_num_pairs(const cascade_tree* tree) { return tree ? tree->n_pairs : 0; }
 int cascade_tree_pairs(const cascade_tree* tree, int32_t* pair_a, int32_t* pair_b) {
   if (tree == nullptr || pair_a == nullptr || pair_b == nullptr) return CASCADE_ERR_INVALID_ARG;
+  if (tree->device_built) {
+    // the list lives on the device only: fetched with blocking copies (the caller has synchronised the stream
+    // of the update); entries beyond the tree's pair count are -1
+    int32_t meta[4] = {0, 0, 0, 0};
+    CASCADE_CUDA_TRY(cudaMemcpy(meta, tree->d_meta, sizeof(meta), cudaMemcpyDeviceToHost));
+    const int n = meta[0] < tree->n_pairs ? meta[0] : tree->n_pairs;
+    CASCADE_CUDA_TRY(cudaMemcpy(pair_a, tree->d_pair_a, sizeof(int32_t) * n, cudaMemcpyDeviceToHost));
+    CASCADE_CUDA_TRY(cudaMemcpy(pair_b, tree->d_pair_b, sizeof(int32_t) * n, cudaMemcpyDeviceToHost));
+    for (int i = n; i < tree->n_pairs; ++i) pair_a[i] = pair_b[i] = -1;
+    return CASCADE_OK;
+  }
   std::memcpy(pair_a, tree->pair_a.data(), sizeof(int32_t) * tree->n_pairs);
   std::memcpy(pair_b, tree->pair_b.data(), sizeof(int32_t) * tree->n_pairs);
   return CASCADE_OK;

@@ -35,7 +35,7 @@ enum KernelId : int {
   K_TREE_ATTN = 0, K_TREE_ATTN_F32, K_FINAL_NORM_MIX, K_GEMM_HEAD, K_HEAD_F32, K_ROW_STATS,
   K_ROW_LSE, K_SIMILARITY, K_ACCEPT, K_TAIL, K_SELECT_PATH, K_EMBED_NORM, K_GEMM_QKV, K_ROPE_SPLIT, K_GEMM_O,
   K_RESID_NORM, K_GEMM_GATE_UP, K_SWIGLU, K_GEMM_DOWN, K_GEMM_F32, K_RESID_ADD, K_KV_APPEND, K_BONUS_TOKEN,
-  K_FILTER_LOGITS, K_WAIT_PROBE, K_KERNEL_ID_END
+  K_FILTER_LOGITS, K_WAIT_PROBE, K_BUILD_TREE, K_KERNEL_ID_END
 };
 static_assert(K_KERNEL_ID_END <= CASCADE_KERNEL_COUNT, "timing table too small");
 
@@ -45,7 +45,7 @@ struct TimedLaunch {
 };
 
 // Bits of the device error word.
-enum : int { CASCADE_DEV_ERR_WAIT = 1, CASCADE_DEV_ERR_OVERFLOW = 2 };
+enum : int { CASCADE_DEV_ERR_WAIT = 1, CASCADE_DEV_ERR_OVERFLOW = 2, CASCADE_DEV_ERR_BAD_TREE = 4 };
 
 struct cascade_ctx {
   cascade_shape shape;
@@ -143,6 +143,10 @@ struct cascade_tree {
   int32_t* d_pair_a = nullptr;
   int32_t* d_pair_b = nullptr;
   uint64_t* d_anc = nullptr;         // [T][4] ancestor-or-self bitmask
+  int32_t* d_meta = nullptr;         // [4] written by the device-side builder: pair count, depth, valid
+  // true after cascade_tree_update_device: the host then knows only T and the caller's bounds -- depth_max is the
+  // depth bound, n_pairs the pair bound (the row length of scores arrays) -- and its mirrors of the arrays are stale
+  bool device_built = false;
 };
 
 // Brackets one kernel launch with events when timing is on; always counts the launch.
@@ -244,6 +248,10 @@ int launch_head_f32(cascade_ctx* ctx, const cascade_tree* tree, const float* w_h
 // The row log-sum-exp is folded from the partials by launch_tail.
 int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bfloat16* w_head,
                      const int32_t* tok, float* logits, float* cand_parent, float* cand_gparent, cudaStream_t s);
+
+// tree_build.cu: the descriptor's device arrays from a device-resident parent[]
+int launch_build_tree(cascade_ctx* ctx, cascade_tree* tree, int T, int depth_cap, int pairs_cap,
+                      const int32_t* parent_dev, cudaStream_t s);
 
 // layer.cu: the decoder layers of a verification step; leaves the residual stream in ctx->x.
 // `pending`: the last MLP output, still to be added to ctx->x by whoever reads it next (empty if the

@@ -51,10 +51,13 @@ __global__ void k_bump_prefix(int B, const int32_t* __restrict__ path_len, int p
   if (prefix_len[r] + n <= prefix_cap) prefix_len[r] += n;
 }
 
-// One CTA per prompt.  Row = logits of the path's end node; the tokens of that node's children (all
-// rejected) get weight zero; token = first v with cumsum(exp(l - max))[v] > u * total.  Every thread owns a
-// contiguous run of the vocabulary; sums in double so that the order of additions does not move the
-// sample.
+// One CTA per prompt.  Row = logits of the path's end node.  Without a drafter row: the tokens of that node's
+// children (all rejected) get weight zero, the others exp(l - max).  With the drafter's distribution p at the end
+// node (draft != null) and at least one rejected child: Algorithm 1's correction step, weight [q - p]+ with
+// q = softmax(l) (and plain q if nothing is left of it, i.e. p >= q everywhere).  After a fully accepted path
+// (the end node has no children) the weight is q's in both modes.  token = first v with cumsum(weight)[v] >
+// u * total.  Every thread owns a contiguous run of the vocabulary; sums in double, runs added in index order,
+// so that the order of additions does not move the sample.
 __global__ void __launch_bounds__(kThreads) k_bonus_token(const float* __restrict__ logits, int T, int V,
                                                           int depth_max, const int32_t* __restrict__ tok,
                                                           const int32_t* __restrict__ child_begin,
@@ -62,6 +65,7 @@ __global__ void __launch_bounds__(kThreads) k_bonus_token(const float* __restric
                                                           const int32_t* __restrict__ path_nodes,
                                                           const int32_t* __restrict__ path_len,
                                                           const float* __restrict__ u_bonus,
+                                                          const float* __restrict__ draft,
                                                           int32_t* __restrict__ token_out,
                                                           float* __restrict__ mass_out) {
   __shared__ int s_rej[CASCADE_MAX_CHILDREN];
@@ -89,7 +93,32 @@ __global__ void __launch_bounds__(kThreads) k_bonus_token(const float* __restric
   __syncthreads();
   m = s_max;
   const int seg = (V + kThreads - 1) / kThreads, v0 = tid * seg, v1 = min(V, v0 + seg);
+  // residual mode needs q itself, i.e. the normaliser of the row, before any weight can be formed
+  const float* p_row = (draft != nullptr && cc > 0) ? draft + (size_t)b * V : nullptr;
+  double inv_z = 0.0;
+  int residual = p_row != nullptr;
+  if (residual) {
+    double z = 0.0;
+    for (int v = v0; v < v1; ++v) z += (double)expf(l[v] - m);
+    s_part[tid] = z;
+    __syncthreads();
+    if (tid == 0) {
+      double run = 0.0;
+      for (int i = 0; i < kThreads; ++i) run += s_part[i];
+      s_total = run;
+    }
+    __syncthreads();
+    inv_z = 1.0 / s_total;
+    // is anything left of q above p?  (not when the drafter's row equals the target's)
+    double r = 0.0;
+    for (int v = v0; v < v1; ++v) r += fmax((double)expf(l[v] - m) * inv_z - (double)p_row[v], 0.0);
+    const int any = __syncthreads_or(r > 0.0);
+    if (!any) residual = 0;
+    __syncthreads();
+  }
   auto weight = [&](int v) {
+    if (residual) return fmax((double)expf(l[v] - m) * inv_z - (double)p_row[v], 0.0);
+    if (p_row != nullptr) return (double)expf(l[v] - m);   // nothing left above p: the target row itself
     for (int c = 0; c < cc; ++c)
       if (s_rej[c] == v) return 0.0;
     return (double)expf(l[v] - m);
@@ -124,7 +153,9 @@ __global__ void __launch_bounds__(kThreads) k_bonus_token(const float* __restric
   __syncthreads();
   if (tid == 0) {
     token_out[b] = s_token;
-    if (mass_out != nullptr) {
+    if (mass_out != nullptr && p_row != nullptr) {
+      mass_out[b] = residual ? (float)total : 1.f;   // sum of [q - p]+: the probability mass the correction keeps
+    } else if (mass_out != nullptr) {
       // remaining mass = total / sum of all weights; the rejected tokens' weights are added back here
       double all = total;
       for (int c = 0; c < cc; ++c) {
@@ -183,8 +214,8 @@ int cascade_kv_append(cascade_ctx* ctx, const cascade_tree* tree, int32_t n_laye
 }
 
 int cascade_bonus_token(cascade_ctx* ctx, const cascade_tree* tree, const float* logits, const int32_t* tok,
-                        const int32_t* path_nodes, const int32_t* path_len, const float* u_bonus, int32_t* token_out,
-                        float* mass_out, void* stream) {
+                        const float* draft_row, const int32_t* path_nodes, const int32_t* path_len,
+                        const float* u_bonus, int32_t* token_out, float* mass_out, void* stream) {
   if (ctx == nullptr || tree == nullptr || logits == nullptr || tok == nullptr || path_nodes == nullptr ||
       path_len == nullptr || u_bonus == nullptr || token_out == nullptr)
     return CASCADE_ERR_INVALID_ARG;
@@ -195,7 +226,7 @@ int cascade_bonus_token(cascade_ctx* ctx, const cascade_tree* tree, const float*
     KernelScope ks(ctx, K_BONUS_TOKEN, s);
     k_bonus_token<<<ctx->shape.B, kThreads, 0, s>>>(logits, tree->T, ctx->shape.V, tree->depth_max, tok,
                                                     tree->d_child_begin, tree->d_child_count, path_nodes, path_len,
-                                                    u_bonus, token_out, mass_out);
+                                                    u_bonus, draft_row, token_out, mass_out);
   }
   CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;

@@ -94,3 +94,74 @@ def test_append_beyond_the_cache_is_refused_not_written():
         loop.step()
     assert e.value.status == cb.ERR_OVERFLOW
     loop.close()
+
+
+def test_residual_draw_of_algorithm_1():
+    """cascade_bonus_token with the drafter's full row at the path's end node: [q - p]+ normalised after a
+    rejection, q after a fully accepted path, q where nothing of q lies above p.  Paths are set by hand so that
+    all three cases occur; many uniforms per case."""
+    from paper_2605_07230_b200.workload import PiecesWorkload
+    w = synth.workload("mini", B=4, tree="topk32", V=4096)
+    wl = PiecesWorkload(w, n_sets=1, keep_logits=True)
+    s = wl.run(0)
+    torch.cuda.synchronize()
+    logits = s.out["logits"].cpu().numpy()
+    parent = wl.parent
+    kids = O.children_of(parent)
+    depth = O.tree_depth(parent)
+    leaf = next(j for j in range(len(parent)) if not kids[j] and depth[j] == wl.tree.depth)
+    inner = next(j for j in range(1, len(parent)) if kids[j])
+    ends = [0, inner, leaf, inner]                       # prompt 3: the drafter's row equals the target's
+    nodes = np.full((w.B, wl.tree.depth + 1), -1, np.int32)
+    plen = np.zeros(w.B, np.int32)
+    for b, end in enumerate(ends):
+        path = []
+        i = end
+        while i >= 0:
+            path.append(i)
+            i = parent[i]
+        path.reverse()
+        nodes[b, : len(path)] = path
+        plen[b] = len(path) - 1
+    rng = np.random.default_rng(23)
+    draft = np.zeros((w.B, w.V), np.float32)
+    for b, end in enumerate(ends):
+        q = O.softmax(logits[b, end].astype(np.float64))
+        if b == 3:
+            draft[b] = q
+            draft[b] = np.maximum(draft[b], q.astype(np.float32) * (1 + 1e-6))   # p >= q everywhere, in fp32 too
+        else:
+            soft = O.softmax(logits[b, end].astype(np.float64) / 1.5 + rng.normal(0, 0.5, w.V))
+            draft[b] = soft
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(G.DEV)
+    d_nodes, d_plen, d_draft = dev(nodes), dev(plen), dev(draft)
+    token = torch.zeros(w.B, dtype=torch.int32, device=G.DEV)
+    mass = torch.zeros(w.B, device=G.DEV)
+    differ = 0
+    for it in range(40):
+        u = rng.random(w.B, dtype=np.float32)
+        cb.cascade_bonus_token(wl.ctx, wl.tree, s.out["logits"], s.dev["tok"], d_nodes, d_plen, dev(u), token, mass,
+                               draft_row=d_draft)
+        torch.cuda.synchronize()
+        got, got_mass = token.cpu().numpy(), mass.cpu().numpy()
+        for b, end in enumerate(ends):
+            want, total = O.residual_token(logits[b, end], draft[b], bool(kids[end]), u[b])
+            assert abs(got_mass[b] - total) < 1e-4, (b, got_mass[b], total)
+            if got[b] != want:
+                # only a draw within 1e-5 of a step of the cumulative distribution may fall to the neighbour
+                qv = O.softmax(logits[b, end].astype(np.float64))
+                wgt = np.maximum(qv - draft[b], 0) if (kids[end] and np.maximum(qv - draft[b], 0).sum() > 0) else qv
+                c = np.cumsum(wgt) / wgt.sum()
+                assert abs(c[min(got[b], want)] - u[b]) < 1e-5, (b, got[b], want)
+                differ += 1
+    assert differ <= 4
+    # without the drafter's row the entry keeps its other rule (children's tokens removed)
+    u = rng.random(w.B, dtype=np.float32)
+    cb.cascade_bonus_token(wl.ctx, wl.tree, s.out["logits"], s.dev["tok"], d_nodes, d_plen, dev(u), token, mass)
+    torch.cuda.synchronize()
+    tok = s.host["tok"]
+    for b, end in enumerate(ends):
+        want, total = O.bonus_token(logits[b, end], [tok[b, c] for c in kids[end]], u[b])
+        assert abs(float(mass[b]) - total) < 1e-4
+    wl.ctx.check()
+    wl.close()

@@ -385,3 +385,83 @@ def test_append_path_kv_writes_the_path_rows_in_order_to_both_cfg_rows():
     assert np.array_equal(k[0, 3:6], kt[0, [0, 2, 4]]) and np.array_equal(k[2, 5:8], kt[2, [0, 2, 4]])
     assert np.array_equal(v[1, 4:5], vt[1, [0]]) and np.array_equal(v[3, 6:7], vt[3, [0]])
     assert k[0, 6:].sum() == 0 and k[1, 5:].sum() == 0
+
+
+# ---- Algorithm 1's correction step: [q - p]+ -------------------------------------------------------------------
+
+
+def _draw_intervals(fn, n_grid=200001):
+    """Lebesgue measure of {u in [0,1) : fn(u) == v} for every v, for a non-decreasing step function fn, found by
+    bisection on its jump points (no sampling): returns {v: measure}."""
+    out = {}
+    lo = 0.0
+    v_lo = fn(lo)
+    while True:
+        hi = 1.0 - 2 ** -53
+        if fn(hi) == v_lo:
+            out[v_lo] = out.get(v_lo, 0.0) + 1.0 - lo
+            return out
+        a, b = lo, hi                        # fn(a) == v_lo, fn(b) != v_lo
+        for _ in range(80):
+            mid = 0.5 * (a + b)
+            if fn(mid) == v_lo:
+                a = mid
+            else:
+                b = mid
+        out[v_lo] = out.get(v_lo, 0.0) + b - lo
+        lo, v_lo = b, fn(b)
+
+
+def test_accept_test_plus_residual_draw_reproduces_the_target_distribution():
+    """The property Section 3 states for Algorithm 1: the emitted token is a sample of the target distribution.
+    One draft position, vocabulary of 7, every quantity exact: the draft x is accepted on the set of u with
+    u < min(1, q(x)/p(x)) (measured on the checker's own accept test with the relaxation off), otherwise the
+    token comes from the residual draw, whose inverse-CDF map is measured interval by interval.
+    sum_x p(x) [ acc(x) delta_x + (1 - acc(x)) res(.) ]  must equal q."""
+    rng = np.random.default_rng(17)
+    V = 7
+    for trial in range(5):
+        logits = rng.normal(0, 1.5, V)
+        q = O.softmax(logits)
+        p = rng.dirichlet(np.ones(V) * 0.7)
+        if trial == 4:
+            p[2] = 0.0                       # a token the drafter never proposes
+            p /= p.sum()
+        res = _draw_intervals(lambda u: O.residual_token(logits, p, True, u)[0])
+        res = np.array([res.get(v, 0.0) for v in range(V)])
+        want_res = np.maximum(q - p, 0)
+        assert np.allclose(res, want_res / want_res.sum(), atol=1e-12)
+        assert abs(O.residual_token(logits, p, True, 0.3)[1] - want_res.sum()) < 1e-15
+        emitted = np.zeros(V)
+        parent = np.array([-1, 0])
+        feat = np.eye(2, 4)
+        for x in range(V):
+            if p[x] == 0:
+                continue
+            def accepted(u):
+                r = O.relaxed_accept(feat, np.stack([logits, logits]), np.array([0, x]), parent,
+                                     np.array([1.0, p[x]]), np.array([0.0, u]), 2.0, 2.0, 0.0, flags=0)
+                return int(r["accept"][1])
+            m = _draw_intervals(accepted)
+            acc = m.get(1, 0.0)
+            assert abs(acc - min(1.0, q[x] / p[x])) < 1e-12
+            emitted[x] += p[x] * acc
+            emitted += p[x] * (1 - acc) * res
+        assert np.allclose(emitted, q, atol=1e-11)
+
+
+def test_residual_draw_special_cases():
+    logits = np.log(np.array([0.1, 0.2, 0.3, 0.4]))
+    q = O.softmax(logits)
+    # nothing rejected: the target row itself, whatever the drafter's row says
+    for u, want in ((0.0, 0), (0.0999, 0), (0.1001, 1), (0.2999, 1), (0.3001, 2), (0.61, 3), (0.999999, 3)):
+        assert O.residual_token(logits, np.array([1.0, 0, 0, 0]), False, u) == (want, 1.0)
+    # drafter = target: nothing lies above p, the target row is used
+    assert O.residual_token(logits, q, True, 0.65)[0] == 3
+    # p takes all of token 3 and more: only tokens where q > p remain, in proportion to the excess
+    p = np.array([0.05, 0.05, 0.1, 0.8])
+    r = np.array([0.05, 0.15, 0.2, 0.0])
+    tok, total = O.residual_token(logits, p, True, 0.51)
+    assert abs(total - r.sum()) < 1e-15 and tok == 2            # cdf 0.125, 0.5, 1.0
+    assert O.residual_token(logits, p, True, 0.49)[0] == 1 and O.residual_token(logits, p, True, 0.12)[0] == 0
+    assert O.residual_token(logits, p, True, 0.999999)[0] == 2  # token 3 has no residual mass
