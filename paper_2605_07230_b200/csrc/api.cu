@@ -55,10 +55,6 @@ int64_t carve(cascade_ctx* c, char* base) {
   cv.take(c->dev_error, 64);
   cv.take(c->gemm_flags, 1024);
   cv.take(c->tail_counters, s.B);
-  const int t_pad = (int)align_up(T, 64);
-  cv.take(c->attn_part_o, (int64_t)R * s.Hq * c->attn_max_splits * t_pad * s.D);
-  cv.take(c->attn_part_ml, (int64_t)R * s.Hq * c->attn_max_splits * t_pad);
-  cv.take(c->attn_unit_done, (int64_t)R * s.Hq * (t_pad / 64));
   c->head_m_pad = (int)align_up(BT, 128);
   if (s.dtype == CASCADE_BF16) {
     cv.take(c->head_a, operand_elems((int)BT, s.h));
@@ -200,11 +196,6 @@ int cascade_create(cascade_ctx** out, const cascade_shape* shape) {
     delete c;
     return CASCADE_ERR_CUDA;
   }
-  // enough KV splits that (rows x kv heads x splits) covers the SMs about twice
-  const int units = 2 * shape->B * shape->Hkv;
-  c->attn_max_splits = ceil_div(2 * c->sm_count, units);
-  if (c->attn_max_splits < 1) c->attn_max_splits = 1;
-  if (c->attn_max_splits > 16) c->attn_max_splits = 16;
   c->ws_bytes = carve(c, nullptr);
   if (cudaMalloc(&c->ws, (size_t)c->ws_bytes) != cudaSuccess) {
     (void)cudaGetLastError();

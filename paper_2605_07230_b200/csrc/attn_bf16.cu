@@ -3,30 +3,57 @@
 // for sm_100a.  Memory-bound decode-style kernel: every key/value row is streamed from HBM once per
 // (CFG row, head) and shared by all tree rows.
 //
-// One CTA per (KV split, query head x row block, CFG row):
+// One CTA per (KV split, query head x 64-row block, CFG row); the splits of one unit form a thread-block cluster.
 //   * two producer threads stream 128-key K tiles and V tiles (bf16, 128-byte swizzle) through their own
 //     rings (2 and 3 slots) and ask the L2 for the tiles after those;
 //   * one thread issues the tensor-core work: S = Q K^T (UMMA 128x128x128) into one of two TMEM score
-//     buffers, and O_tile = P V into one of two TMEM output buffers;
-//   * four softmax warps own the 128 TMEM lanes.  A row block holds at most 64 tree rows, and the
-//     Q tile is loaded twice (UMMA rows r and r+64 are the same tree row): lanes 0-63 take keys 0-63
-//     of every tile and lanes 64-127 take keys 64-127, so all four warps work although there are only
-//     64 rows.  Each lane keeps its own running (max, sum, output[128]) in registers (online softmax in
-//     the exp2 domain); P goes to shared memory as bf16 in the swizzled K-major layout the UMMA reads,
-//     with the other half of each row held at zero.  The two halves of a row are merged once at the end;
+//     buffers, and O += P V into the TMEM output accumulator;
+//   * eight softmax warps own the 128 TMEM lanes twice over.  A row block holds at most 64 tree rows and the Q
+//     tile is loaded twice (UMMA rows r and r+64 are the same tree row), so that lanes 0-63 can take keys 0-63 of
+//     every tile and lanes 64-127 keys 64-127; the two warps that share a lane quadrant split those 64 keys again.
+//     Four threads therefore work on one tree row, 32 keys each;
+//   * the probabilities go to the tensor core as a bf16 pair: the value rounded to bf16 in P rows 0-63 and what the
+//     rounding dropped (again bf16) in P rows 64-127, so that one UMMA over the 128-row P tile accumulates
+//     sum(p_hi v) in output rows 0-63 and sum(p_lo v) in rows 64-127.  Their sum carries 16 significant bits of
+//     every weight instead of 8; a bf16-rounded P alone limits the output to about 2e-3, which one decoder layer
+//     turns into 2e-2 on the logits;
+//   * online softmax in the exp2 domain with ONE reference per tree row, shared by its four threads and raised
+//     lazily: weights are 2^(s - ref), and ref only has to stay within a few dozen binary orders of the true
+//     maximum for fp32 accumulators (the final division removes it).  The first tile fixes ref by an exchange
+//     through shared memory behind one barrier; later a thread that meets a score more than 2^8 above ref posts
+//     it, and all four threads of the row adopt it at the start of the NEXT tile, behind the wait for the
+//     previous output product, where everybody is known to have seen the post.  The rows already accumulated in
+//     TMEM are then rescaled in place (tcgen05.ld/st); this is rare;
 //   * keys of the prefix are visible to every row up to prefix_len; keys of the tree are visible to
-//     row j iff bit i of the packed ancestor-or-self mask of j is set (one 64-bit word per lane and
-//     tile half).
-// With several KV splits each CTA writes an un-normalised partial (output, max, sum); the CTA of a
-// (CFG row, head, row block) that finishes last merges them in split order (a counter per unit, no
-// waiting) and writes the bf16 rows.  With one split the CTA writes the final rows itself.
-// Every mbarrier wait is bounded (error word + normal teardown on expiry).
+//     row j iff bit i of the packed ancestor-or-self mask of j is set.
+// With several KV splits every CTA leaves its un-normalised partial (output rows, reference, sum) in its own shared
+// memory; the rank-0 CTA of the cluster reads the others' through distributed shared memory, merges in split
+// order and writes the rows.  No global scratch, no counters.
+// Every mbarrier wait is bounded (error word + normal teardown on expiry); the cluster barriers at the start and
+// the end are reached by every thread on every path.
 #include "cascade_internal.h"
 #include "operand.cuh"
 #include "ptx.cuh"
 #include "tmap.h"
 
 namespace {
+
+constexpr int kD = 128;
+constexpr int kTileKeys = 128;
+constexpr int kRowsPerBlock = 64;
+constexpr int kSoftmaxThreads = 256;  // warps 0-7
+constexpr int kThreads = 320;         // + warp 8: TMA, warp 9: UMMA issue + TMEM alloc
+constexpr int kQBytes = 128 * kD * 2;        // 32 KB: two 64-wide halves of [128 rows][64] bf16
+constexpr int kPBytes = 128 * kTileKeys * 2;  // 32 KB
+constexpr int kKVTileBytes = kTileKeys * kD * 2;  // 32 KB for K, same for V
+constexpr int kKSlots = 2;     // K tiles in shared memory (a slot is free again once S = Q K^T has read it)
+constexpr int kVSlots = 3;     // V tiles in shared memory (free once O += P V has read it)
+constexpr int kPrefetch = 0;   // with a ring of n slots, tile i + n - 1 + kPrefetch is requested into the L2 when tile i is
+                               // loaded (measured 0..3 on 20-tile rows: deeper requests delay the loads that are waited for)
+constexpr int kSmemBytes = kQBytes + kPBytes + (kKSlots + kVSlots) * kKVTileBytes + 1024;
+constexpr int kXRow = 132;     // floats per row of the partial-result buffer: 128 outputs, reference, sum, 2 pad
+constexpr int kMaxSplits = 4;
+constexpr float kLazy = 8.f;   // the reference is raised when a score exceeds it by more than this (log2 units)
 
 // 8 consecutive outputs of (row m of R*T, column col of Hq*D): bf16 row-major, or -- for the output
 // projection that follows inside a decoder layer -- the bf16 pair (value, what the rounding dropped) in the
@@ -47,35 +74,24 @@ __device__ __forceinline__ void store8(const Args& p, int m, int col, int row_le
   }
 }
 
-constexpr int kD = 128;
-constexpr int kTileKeys = 128;
-constexpr int kRowsPerBlock = 64;
-constexpr int kThreads = 192;  // warps 0-3 softmax, warp 4 TMA, warp 5 UMMA issue + TMEM alloc
-constexpr int kQBytes = 128 * kD * 2;        // 32 KB: two 64-wide halves of [128 rows][64] bf16
-constexpr int kPBytes = 128 * kTileKeys * 2;  // 32 KB
-constexpr int kKVTileBytes = kTileKeys * kD * 2;  // 32 KB for K, same for V
-constexpr int kKSlots = 2;     // K tiles in shared memory (a slot is free again once S = Q K^T has read it)
-constexpr int kVSlots = 3;     // V tiles in shared memory (free once O += P V has read it)
-constexpr int kPrefetch = 0;   // with a ring of n slots, tile i + n - 1 + kPrefetch is requested into the L2 when tile i is
-                               // loaded (measured 0..3 on 20-tile rows: deeper requests delay the loads that are waited for)
-constexpr int kSmemBytes = kQBytes + kPBytes + (kKSlots + kVSlots) * kKVTileBytes + 1024;
-constexpr int kXRow = 132;  // row stride (floats) of the half-merge exchange buffer (16-byte aligned rows)
-constexpr int kORow = 132;  // row stride (floats) of the output staging buffer (16-byte aligned rows)
-
 struct AttnArgs {
-  int T, Hq, Hkv, splits, n_rb, t_pad, prefix_cap;
+  int T, Hq, Hkv, splits, n_rb, prefix_cap;
   const int32_t* prefix_len;
   const uint64_t* anc;
   __nv_bfloat16* out;
   int out_as_operand;     // 1: `out` receives the (R*T x Hq*D) matrix as a GEMM operand (bf16 pair, staged layout)
   OperandLayout out_lay;
-  float* part_o;
-  float2* part_ml;
   float c;  // softmax_scale * log2(e)
   int* err;
   unsigned long long wait_ns;  // limit of every bounded wait in the kernel
-  unsigned int* unit_done;  // [R * Hq * n_rb] finished-split counters, zero between launches
 };
+
+// order-preserving image of a float in a signed int (for atomicMax on shared memory)
+__device__ __forceinline__ int float_key(float f) {
+  const int b = __float_as_int(f);
+  return b >= 0 ? b : b ^ 0x7fffffff;
+}
+__device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kp,
@@ -83,9 +99,10 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                  const __grid_constant__ CUtensorMap tm_vt, const AttnArgs p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t q_full, k_full[kKSlots], k_empty[kKSlots], v_full[kVSlots], v_empty[kVSlots],
-      s_full[2], s_empty[2], p_full, o_full;
+      s_full[2], s_empty[2], p_full, o_full, ref_ready, peers_ready;
   __shared__ uint32_t s_tmem_base;
-  __shared__ int s_abort, s_last;
+  __shared__ int s_abort;
+  __shared__ int s_rowmax[3][kRowsPerBlock];   // posted row maxima, one buffer per tile index mod 3
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -93,7 +110,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t q_addr = smem_base, p_addr = smem_base + kQBytes, k_ring = p_addr + kPBytes,
                  v_ring = k_ring + kKSlots * kKVTileBytes;
 
-  if (threadIdx.x == 128) {  // the TMA warp's first loads should not wait for their descriptors
+  if (threadIdx.x == kSoftmaxThreads) {  // the TMA warp's first loads should not wait for their descriptors
     ptx::prefetch_tmap(&tm_q);
     ptx::prefetch_tmap(&tm_kp);
     ptx::prefetch_tmap(&tm_vp);
@@ -106,9 +123,13 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int n_ptiles = (P + kTileKeys - 1) / kTileKeys;
   const int n_ttiles = (p.T + kTileKeys - 1) / kTileKeys;
   const int total = n_ptiles + n_ttiles;
-  const int per = (total + p.splits - 1) / p.splits;
-  const int tile_begin = split * per;
-  const int tile_end = min(total, tile_begin + per);
+  // the tiles of the tree's own keys stay in one split (they count as one item of the division), so that in every
+  // CTA a row either sees a key in the CTA's first tile or in none of its tiles
+  const int items = n_ptiles + 1;
+  const int per = (items + p.splits - 1) / p.splits;
+  const int tile_begin = min(split * per, items);
+  const int item_end = min(items, tile_begin + per);
+  const int tile_end = item_end == items ? total : item_end;
   const int n = max(0, tile_end - tile_begin);
 
   if (threadIdx.x == 0) {
@@ -123,35 +144,37 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&s_full[i], 1);
-      ptx::mbar_init(&s_empty[i], 128);
+      ptx::mbar_init(&s_empty[i], kSoftmaxThreads);
     }
-    ptx::mbar_init(&p_full, 128);
+    ptx::mbar_init(&p_full, kSoftmaxThreads);
     ptx::mbar_init(&o_full, 1);
+    ptx::mbar_init(&ref_ready, kSoftmaxThreads);
+    ptx::mbar_init(&peers_ready, max(1, p.splits - 1));
     s_abort = 0;
     ptx::fence_mbar_init();
   }
+  if (threadIdx.x < 3 * kRowsPerBlock) (&s_rowmax[0][0])[threadIdx.x] = float_key(-INFINITY);
   __syncthreads();  // barriers are initialised: the producers start streaming at once
+  ptx::cluster_arrive();  // ... and the other CTAs of the cluster may signal this one once they have seen this
   volatile int* abort_flag = &s_abort;
-  if (warp != 4) {
-    // meanwhile the other warps zero P (each UMMA row only ever writes its own key half) and get TMEM
-    for (int i = warp == 5 ? 128 + lane : threadIdx.x; i < kPBytes / 16; i += 160)
-      reinterpret_cast<uint4*>(smem + kQBytes)[i] = make_uint4(0, 0, 0, 0);
-    ptx::fence_proxy_async_smem();
-    if (warp == 5) {
+  if (warp != 8) {
+    if (warp == 9) {
       ptx::tmem_alloc(&s_tmem_base, 512);
       ptx::tmem_relinquish();
     }
     ptx::tc_fence_before();
-    ptx::named_bar_sync(2, 160);
+    ptx::named_bar_sync(2, kThreads - 32);
     ptx::tc_fence_after();
   }
-  const uint32_t tmem_base = warp != 4 ? s_tmem_base : 0u;
+  const uint32_t tmem_base = warp != 8 ? s_tmem_base : 0u;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
+  float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);  // partial result, in the K ring once the loop is over
+  // small arrays of the end phase, in the Q tile's place (idle once the last scores have been issued)
+  float (*s_lsum)[kRowsPerBlock] = reinterpret_cast<float (*)[kRowsPerBlock]>(smem);          // [4]: a row's four partial sums
+  float (*s_w)[kRowsPerBlock] = reinterpret_cast<float (*)[kRowsPerBlock]>(smem + 1024);      // [kMaxSplits]: merge weights
+  float* s_inv = reinterpret_cast<float*>(smem + 1024 + kMaxSplits * kRowsPerBlock * 4);
 
-  // softmax state (warps 0-3)
-  float m_run = -INFINITY, l_run = 0.f;
-
-  if (warp == 4) {
+  if (warp == 8) {
     // ---------------- TMA producers: lane 0 streams Q and the K tiles, lane 1 the V tiles ----------------
     // The rings hold less than HBM latency x this SM's share of the bandwidth, so tiles further ahead
     // are also requested into the L2.
@@ -211,7 +234,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (t < n) prefetch_tile(t);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ---------------- UMMA issue ----------------
     // S(i) = Q K_i^T needs K tile i and a free score buffer; O += P_i V_i needs the softmax of tile i and
     // V tile i.  Whichever is ready is issued, so scores run ahead of the softmax while the output product
@@ -283,120 +306,149 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
   } else {
     // ---------------- softmax warps ----------------
-    const int urow = warp * 32 + lane;        // UMMA row == TMEM lane
-    const int row_in_block = urow & 63;
-    const int khalf = urow >> 6;              // which 64 keys of each tile this lane owns
-    const int j = rb * kRowsPerBlock + row_in_block;  // tree row
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    const int quad = warp & 3, sub = warp >> 2;   // TMEM lane quadrant; which 32 of the quadrant's 64 keys
+    const int row = (quad & 1) * 32 + lane;       // tree row within the block; TMEM lanes row and row + 64 belong to it
+    const int kofs = (quad >> 1) * 64 + sub * 32; // first key (within a tile) of this thread's 32
+    const int j = rb * kRowsPerBlock + row;       // tree row
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint64_t anc_w[4] = {0, 0, 0, 0};
     if (j < p.T) {
 #pragma unroll
       for (int w = 0; w < 4; ++w) anc_w[w] = p.anc[(size_t)j * 4 + w];
     }
-    const uint32_t p_row_addr = p_addr + khalf * (128 * 128) + urow * 128;
-    const uint32_t o_addr = tmem_o + lane_addr;
-    // Online softmax with a lazily updated reference: weights are 2^(s - m_run) where m_run is only
-    // raised when a tile's maximum exceeds it by more than kLazy (so weights stay below 2^kLazy).
-    // The outputs then accumulate across tiles inside TMEM (the UMMA adds into O); this lane's O and
-    // sum are rescaled only on the rare tile that raises m_run.
-    constexpr float kLazy = 8.f;
+    // P rows `row` (bf16 value) and `row + 64` (remainder); this thread's 32 keys are 4 pieces of 16 bytes in the
+    // 64-key column block (quad >> 1), at piece positions 4 sub .. 4 sub + 3 before the swizzle
+    const uint32_t p_hi_row = p_addr + (quad >> 1) * (128 * 128) + row * 128;
+    const uint32_t p_lo_row = p_hi_row + 64 * 128;
+    const uint32_t o_cols = tmem_o + lane_addr + sub * 64;  // the 64 output columns this thread rescales / reads
+    float m_ref = -INFINITY;   // the row's reference (same value in the row's four threads)
+    float l_run = 0.f;         // sum of this thread's weights
     bool ok = n > 0;
     for (int i = 0; ok && i < n; ++i) {
       if (!ptx::mbar_wait(&s_full[i & 1], (i >> 1) & 1u, abort_flag, p.err, p.wait_ns)) { ok = false; break; }
       ptx::tc_fence_after();
       const int tile = tile_begin + i;
       const bool in_prefix = tile < n_ptiles;
-      const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys + khalf * 64;
-      // visibility of this lane's 64 keys as one 64-bit word (rows beyond T see the prefix like any other:
-      // their query is the zero fill of the tensor map and nothing of theirs is ever stored; that keeps the
-      // test below uniform over a warp)
-      uint64_t vis;
+      const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys + kofs;
+      // visibility of this thread's 32 keys (rows beyond T see the prefix like any other: their query is the
+      // zero fill of the tensor map and nothing of theirs is ever stored; that keeps the test below uniform)
+      uint32_t vis;
       if (in_prefix) {
         const int nvis = P - key0;
-        vis = nvis <= 0 ? 0ull : (nvis >= 64 ? ~0ull : ((1ull << nvis) - 1ull));
+        vis = nvis <= 0 ? 0u : (nvis >= 32 ? ~0u : ((1u << nvis) - 1u));
       } else {
-        vis = anc_w[(key0 >> 6) & 3];
+        vis = (uint32_t)(anc_w[(key0 >> 6) & 3] >> (key0 & 63));
       }
-      float sc[64];
-      ptx::tmem_ld64(tmem_s + lane_addr + (i & 1) * 128 + khalf * 64, sc);
+      float sc[32];
+      ptx::tmem_ld32(tmem_s + lane_addr + (i & 1) * 128 + kofs, sc);
       ptx::tc_fence_before();
       ptx::mbar_arrive(&s_empty[i & 1]);
       // A tile every row of the warp sees whole (all but the last prefix tile) needs no masking, and with a
-      // positive scale the maximum can be taken before scaling: weight = 2^(s * c - m) in one multiply-add.
-      const bool whole = p.c > 0.f && __all_sync(0xffffffffu, vis == ~0ull);
+      // positive scale the maximum can be taken before scaling: weight = 2^(s * c - ref) in one multiply-add.
+      const bool whole = p.c > 0.f && __all_sync(0xffffffffu, vis == ~0u);
       float m_tile = -INFINITY;
       if (whole) {
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int k = 0; k < 64; ++k) m4[k & 3] = fmaxf(m4[k & 3], sc[k]);
+        for (int k = 0; k < 32; ++k) m4[k & 3] = fmaxf(m4[k & 3], sc[k]);
         m_tile = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * p.c;
       } else {
 #pragma unroll
-        for (int k = 0; k < 64; ++k) {
-          sc[k] = ((vis >> k) & 1ull) ? sc[k] * p.c : -INFINITY;
+        for (int k = 0; k < 32; ++k) {
+          sc[k] = ((vis >> k) & 1u) ? sc[k] * p.c : -INFINITY;
           m_tile = fmaxf(m_tile, sc[k]);
         }
       }
       const float mul = whole ? p.c : 1.f;  // the masked path has scaled its scores already
-      float alpha = 1.f;  // factor for what this lane has accumulated so far
-      if (m_run == -INFINITY) {
-        m_run = m_tile;   // nothing accumulated yet (all weights so far were zero)
-      } else if (m_tile > m_run + kLazy) {
-        alpha = ptx::ex2(m_run - m_tile);
-        m_run = m_tile;
+      if (i == 0) {
+        // the first tile fixes the row's reference: the maximum over its four threads
+        if (m_tile != -INFINITY) atomicMax(&s_rowmax[0][row], float_key(m_tile));
+        ptx::mbar_arrive(&ref_ready);
+        if (!ptx::mbar_wait(&ref_ready, 0, abort_flag, p.err, p.wait_ns)) { ok = false; break; }
+        m_ref = key_float(s_rowmax[0][row]);
+      } else if (m_tile > m_ref + kLazy) {
+        atomicMax(&s_rowmax[i % 3][row], float_key(m_tile));  // adopted by the whole row at the next tile
       }
-      const float m_use = m_run == -INFINITY ? 0.f : m_run;
+      const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
       float rowsum = 0.f;
-      uint32_t packed[32];
 #pragma unroll
-      for (int k = 0; k < 64; k += 2) {
-        const float p0 = ptx::ex2(fmaf(sc[k], mul, -m_use)), p1 = ptx::ex2(fmaf(sc[k + 1], mul, -m_use));
-        packed[k >> 1] = ptx::pack_bf16x2(p0, p1);
-        // sum what the tensor core will actually see (bf16-rounded) so that weights add up to one
-        rowsum += __uint_as_float(packed[k >> 1] << 16) + __uint_as_float(packed[k >> 1] & 0xffff0000u);
+      for (int k = 0; k < 32; ++k) {
+        sc[k] = ptx::ex2(fmaf(sc[k], mul, -m_use));
+        rowsum += sc[k];
+      }
+      if (!(rowsum < 1e37f)) {
+        // a score more than 2^120 above everything the row met in earlier tiles (the reference follows with one
+        // tile's delay): weights are capped at 2^120 instead of overflowing.  What came before is then below
+        // 2^-96 of the result either way.
+        rowsum = 0.f;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+          sc[k] = fminf(sc[k], 1.329228e36f);
+          rowsum += sc[k];
+        }
       }
       if (i >= 1) {
-        // PV(i-1) complete: P may be overwritten and O holds tiles 0..i-1
+        // PV(i-1) complete: P may be overwritten, O holds tiles 0..i-1, and every post of tile i-1 is visible
         if (!ptx::mbar_wait(&o_full, (i - 1) & 1u, abort_flag, p.err, p.wait_ns)) { ok = false; break; }
+        const float posted = key_float(s_rowmax[(i - 1) % 3][row]);
+        float alpha = 1.f;
+        if (posted > m_ref + kLazy) {   // the same decision in all four threads of the row
+          alpha = m_ref == -INFINITY ? 0.f : ptx::ex2(m_ref - posted);
+          m_ref = posted;
+        }
         if (__any_sync(0xffffffffu, alpha != 1.f)) {
+          // rare: this tile's weights and what has been accumulated so far move to the new reference
+#pragma unroll
+          for (int k = 0; k < 32; ++k) sc[k] *= alpha;
+          rowsum *= alpha;
+          l_run *= alpha;
           ptx::tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
+          for (int c = 0; c < 4; ++c) {
             float t[16];
-            ptx::tmem_ld16(o_addr + c * 16, t);
+            ptx::tmem_ld16(o_cols + c * 16, t);
 #pragma unroll
             for (int k = 0; k < 16; ++k) t[k] *= alpha;
-            ptx::tmem_st16(o_addr + c * 16, t);
+            ptx::tmem_st16(o_cols + c * 16, t);
           }
           ptx::tc_fence_before();
         }
       }
+      // the bf16 value and what its rounding dropped, four 16-byte pieces each
 #pragma unroll
-      for (int c = 0; c < 8; ++c)
-        ptx::st_shared_v4(p_row_addr + ((c ^ (urow & 7)) << 4), packed[4 * c], packed[4 * c + 1], packed[4 * c + 2],
-                          packed[4 * c + 3]);
+      for (int c = 0; c < 4; ++c) {
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float a = sc[8 * c + 2 * k], b = sc[8 * c + 2 * k + 1];
+          hi[k] = ptx::pack_bf16x2(a, b);
+          lo[k] = ptx::pack_bf16x2(a - __uint_as_float(hi[k] << 16), b - __uint_as_float(hi[k] & 0xffff0000u));
+        }
+        const uint32_t piece = (uint32_t)((4 * sub + c) ^ (row & 7)) << 4;
+        ptx::st_shared_v4(p_hi_row + piece, hi[0], hi[1], hi[2], hi[3]);
+        ptx::st_shared_v4(p_lo_row + piece, lo[0], lo[1], lo[2], lo[3]);
+      }
       ptx::fence_proxy_async_smem();
       ptx::mbar_arrive(&p_full);
-      l_run = l_run * alpha + rowsum;
+      l_run += rowsum;
     }
     // The code from here to the end of the kernel runs once per CTA from a cold instruction cache, where
     // every instruction line costs a fetch of its own: loops are rolled and the accumulator is taken from
-    // TMEM 16 columns at a time instead of as 128 registers.
+    // TMEM 16 columns at a time.
     bool have_o = false;
     if (ok && n > 0) have_o = ptx::mbar_wait(&o_full, (n - 1) & 1u, abort_flag, p.err, p.wait_ns);
     have_o = __all_sync(0xffffffffu, have_o);  // the TMEM loads below are warp-wide
     ptx::tc_fence_after();
-    // ---- merge the two key halves of each row (lanes r and r+64), then write ----
-    // all UMMAs and TMA copies of this CTA have completed: the KV ring is free to reuse
-    float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);  // the K ring: 64 rows x kXRow floats fit
-    ptx::named_bar_sync(1, 128);
-    if (khalf == 1) {
-      float* x = xbuf + row_in_block * kXRow;
+    // All UMMAs and TMA copies of this CTA have completed: the K ring is free to hold the partial result.
+    // Rows 64-127 of the accumulator (the remainders' share) go to the buffer first, rows 0-63 are added to them.
+    ptx::named_bar_sync(1, kSoftmaxThreads);
+    float* x = xbuf + row * kXRow + sub * 64;
+    if (quad >= 2) {
 #pragma unroll 1
-      for (int c = 0; c < kD / 16; ++c) {
+      for (int c = 0; c < 4; ++c) {
         float v[16];
         if (have_o) {
-          ptx::tmem_ld16(o_addr + 16 * c, v);
+          ptx::tmem_ld16(o_cols + 16 * c, v);
         } else {
 #pragma unroll
           for (int k = 0; k < 16; ++k) v[k] = 0.f;
@@ -405,169 +457,117 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
         for (int k = 0; k < 4; ++k) dst[k] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
       }
-      x[kD] = m_run;
-      x[kD + 1] = l_run;
     }
-    ptx::named_bar_sync(1, 128);
-    // Rows leave through shared memory: a thread holds a whole row here, and writing it directly would put
-    // 16 bytes per lane 512 bytes apart (measured: 5 us for 32 KB).  The Q / P area is idle by now.
-    float* obuf = reinterpret_cast<float*>(smem);  // [64 rows][kORow floats]
-    if (khalf == 0) {
-      const float* x = xbuf + row_in_block * kXRow;
-      const float m1 = x[kD], l1 = x[kD + 1];
-      const float m = fmaxf(m_run, m1);
-      float w0 = m_run == -INFINITY ? 0.f : ptx::ex2(m_run - m);
-      float w1 = m1 == -INFINITY ? 0.f : ptx::ex2(m1 - m);
-      const float l = l_run * w0 + l1 * w1;
-      if (p.splits == 1) {  // final values
-        const float inv = 1.f / l;
-        w0 *= inv;
-        w1 *= inv;
-      } else if (j < p.T) {
-        const size_t unit = ((size_t)r * p.Hq + head) * p.splits + split;
-        p.part_ml[unit * p.t_pad + j] = make_float2(m, l);
-      }
-      float* orow = obuf + row_in_block * kORow;
+    s_lsum[(quad >> 1) * 2 + sub][row] = l_run;
+    ptx::named_bar_sync(1, kSoftmaxThreads);
+    if (quad < 2) {
 #pragma unroll 1
-      for (int c = 0; c < kD / 16; ++c) {
+      for (int c = 0; c < 4; ++c) {
         float v[16];
         if (have_o) {
-          ptx::tmem_ld16(o_addr + 16 * c, v);
+          ptx::tmem_ld16(o_cols + 16 * c, v);
         } else {
 #pragma unroll
           for (int k = 0; k < 16; ++k) v[k] = 0.f;
         }
-        if (j < p.T) {
+        float4* dst = reinterpret_cast<float4*>(x + 16 * c);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const float4 xv = *reinterpret_cast<const float4*>(x + 16 * c + 4 * k);
-            *reinterpret_cast<float4*>(orow + 16 * c + 4 * k) =
-                make_float4(v[4 * k] * w0 + xv.x * w1, v[4 * k + 1] * w0 + xv.y * w1, v[4 * k + 2] * w0 + xv.z * w1,
-                            v[4 * k + 3] * w0 + xv.w * w1);
-          }
+        for (int k = 0; k < 4; ++k) {
+          const float4 lo = dst[k];
+          dst[k] = make_float4(v[4 * k] + lo.x, v[4 * k + 1] + lo.y, v[4 * k + 2] + lo.z, v[4 * k + 3] + lo.w);
         }
+      }
+      if (sub == 0) {   // the row's reference and the sum of its weights ride behind its 128 outputs
+        xbuf[row * kXRow + kD] = m_ref;
+        xbuf[row * kXRow + kD + 1] = s_lsum[0][row] + s_lsum[1][row] + s_lsum[2][row] + s_lsum[3][row];
       }
     }
     ptx::tc_fence_before();
-    ptx::named_bar_sync(1, 128);
-    if (p.splits == 1) {
-      // 16 pieces of 8 outputs per row; consecutive lanes take consecutive pieces (rolled: run-once code)
+  }
+  // ---- splits: rank 0 of the cluster collects the partial results of the others ----
+  // (measured against sharing the rows between the CTAs, each reading its rows of every partial: loads from
+  // another CTA's shared memory are slow enough that one reader of all rows finishes a microsecond sooner)
+  const uint32_t rank = ptx::cluster_ctarank();
+  __syncwarp();
+  ptx::cluster_wait();   // every CTA of the cluster has initialised its barriers (arrived right after doing so)
+  __syncthreads();       // ... and this CTA's partial result is complete for every thread to see
+  if (p.splits > 1 && rank != 0 && threadIdx.x == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&peers_ready), 0));
+  if (warp < 8 && (p.splits == 1 || rank == 0)) {
+    bool merged_ok = true;
+    if (p.splits > 1) merged_ok = ptx::mbar_wait_cluster(&peers_ready, 0, abort_flag, p.err, p.wait_ns);
+    merged_ok = __all_sync(0xffffffffu, merged_ok);
+    // weights of the splits per row: out = sum_s w_s O_s / sum_s w_s l_s, w_s = 2^(ref_s - max ref), in split order
+    const uint32_t x_addr = ptx::smem_u32(xbuf);
+    if (threadIdx.x < kRowsPerBlock) {
+      const int rw = threadIdx.x;
+      float ms[kMaxSplits], ls[kMaxSplits], m = -INFINITY;
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s) {
+        ms[s] = -INFINITY;
+        ls[s] = 0.f;
+        if (s == 0) {
+          ms[s] = xbuf[rw * kXRow + kD];
+          ls[s] = xbuf[rw * kXRow + kD + 1];
+        } else if (s < p.splits && merged_ok) {
+          const uint32_t a = ptx::map_to_cta(x_addr + (uint32_t)(rw * kXRow + kD) * 4u, (uint32_t)s);
+          ms[s] = ptx::ld_cluster_f32(a);
+          ls[s] = ptx::ld_cluster_f32(a + 4u);
+        }
+        m = fmaxf(m, ms[s]);
+      }
+      float l = 0.f;
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s) {
+        const float w = ms[s] == -INFINITY ? 0.f : ptx::ex2(ms[s] - m);
+        s_w[s][rw] = w;
+        l += w * ls[s];
+      }
+      s_inv[rw] = 1.f / l;
+    }
+    ptx::named_bar_sync(1, kSoftmaxThreads);
+    // 16 pieces of 8 outputs per row; consecutive threads take consecutive pieces (rolled: run-once code)
 #pragma unroll 1
-      for (int i = 0; i < 8; ++i) {
-        const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
-        const int jj = rb * kRowsPerBlock + row;
-        if (jj < p.T) {
-          const float4 a = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8);
-          const float4 b = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8 + 4);
-          const float v8[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-          store8(p, r * p.T + jj, head * kD + piece * 8, p.Hq * kD, v8);
+    for (int i = 0; i < 4; ++i) {
+      const int idx = i * kSoftmaxThreads + (int)threadIdx.x, rw = idx >> 4, piece = idx & 15;
+      const int jj = rb * kRowsPerBlock + rw;
+      if (jj >= p.T) continue;
+      const uint32_t off = (uint32_t)(rw * kXRow + piece * 8) * 4u;
+      float4 a = *reinterpret_cast<const float4*>(xbuf + rw * kXRow + piece * 8);
+      float4 b = *reinterpret_cast<const float4*>(xbuf + rw * kXRow + piece * 8 + 4);
+      const float w0 = s_w[0][rw];
+      float acc[8] = {a.x * w0, a.y * w0, a.z * w0, a.w * w0, b.x * w0, b.y * w0, b.z * w0, b.w * w0};
+      if (merged_ok) {
+        for (int s = 1; s < p.splits; ++s) {
+          const uint32_t ra = ptx::map_to_cta(x_addr + off, (uint32_t)s);
+          a = ptx::ld_cluster_v4(ra);
+          b = ptx::ld_cluster_v4(ra + 16u);
+          const float w = s_w[s][rw];
+          acc[0] += w * a.x;
+          acc[1] += w * a.y;
+          acc[2] += w * a.z;
+          acc[3] += w * a.w;
+          acc[4] += w * b.x;
+          acc[5] += w * b.y;
+          acc[6] += w * b.z;
+          acc[7] += w * b.w;
         }
       }
-    } else {
-      const size_t unit = ((size_t)r * p.Hq + head) * p.splits + split;
-#pragma unroll 2
-      for (int i = 0; i < 16; ++i) {
-        const int idx = i * 128 + (int)threadIdx.x, row = idx >> 5, c4 = idx & 31;
-        const int jj = rb * kRowsPerBlock + row;
-        if (jj < p.T)
-          *reinterpret_cast<float4*>(p.part_o + (unit * p.t_pad + jj) * kD + 4 * c4) =
-              *reinterpret_cast<const float4*>(obuf + row * kORow + 4 * c4);
-      }
+      const float inv = s_inv[rw];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] *= inv;
+      store8(p, r * p.T + jj, head * kD + piece * 8, p.Hq * kD, acc);
     }
   }
   __syncwarp();
   __syncthreads();
   if (*abort_flag) __nanosleep(500000);
-  if (warp == 5) {
+  if (warp == 9) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, 512);
   }
-  if (p.splits == 1) return;
-  // ---- the last split of this (CFG row, head, row block) to finish merges all of them ----
-  const unsigned int unit_id = ((unsigned)r * p.Hq + head) * p.n_rb + rb;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const unsigned int ticket = atomicAdd(p.unit_done + unit_id, 1u);
-    s_last = ticket == (unsigned)p.splits - 1;
-    if (s_last) p.unit_done[unit_id] = 0u;
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  if (threadIdx.x >= 128) return;
-  // out = sum_s w_s O_s / sum_s w_s l_s, w_s = 2^(m_s - max m), splits taken in index order.  The weights of a
-  // row go through shared memory, so that consecutive lanes can take consecutive 32-byte pieces of the
-  // partial outputs (a row per lane would read 16 bytes every 512).
-  const size_t unit0 = ((size_t)r * p.Hq + head) * p.splits;
-  float* s_w = reinterpret_cast<float*>(smem);  // [splits][64] weights, then [64] 1 / sum
-  float* s_inv = s_w + p.splits * kRowsPerBlock;
-  if (threadIdx.x < kRowsPerBlock) {
-    const int row = threadIdx.x, jj = rb * kRowsPerBlock + row;
-    if (jj < p.T) {
-      float m = -INFINITY;
-      for (int s = 0; s < p.splits; ++s) m = fmaxf(m, __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + jj]).x);
-      float l = 0.f;
-      for (int s = 0; s < p.splits; ++s) {
-        const float2 ml = __ldcg(&p.part_ml[(unit0 + s) * p.t_pad + jj]);
-        const float w = ml.x == -INFINITY ? 0.f : ptx::ex2(ml.x - m);
-        s_w[s * kRowsPerBlock + row] = w;
-        l += w * ml.y;
-      }
-      s_inv[row] = 1.f / l;
-    }
-  }
-  ptx::named_bar_sync(1, 128);
-  float acc[8][8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int k = 0; k < 8; ++k) acc[i][k] = 0.f;
-  for (int s = 0; s < p.splits; ++s) {
-    float4 t[8][2];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {  // every load of this split issued before the first use
-      const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
-      const int jj = min(rb * kRowsPerBlock + row, p.T - 1);
-      const float4* src = reinterpret_cast<const float4*>(p.part_o + ((unit0 + s) * p.t_pad + jj) * kD + piece * 8);
-      t[i][0] = __ldcg(src);
-      t[i][1] = __ldcg(src + 1);
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float w = s_w[s * kRowsPerBlock + ((i * 128 + (int)threadIdx.x) >> 4)];
-      acc[i][0] += w * t[i][0].x;
-      acc[i][1] += w * t[i][0].y;
-      acc[i][2] += w * t[i][0].z;
-      acc[i][3] += w * t[i][0].w;
-      acc[i][4] += w * t[i][1].x;
-      acc[i][5] += w * t[i][1].y;
-      acc[i][6] += w * t[i][1].z;
-      acc[i][7] += w * t[i][1].w;
-    }
-  }
-  // The sums go back to shared memory and leave through a short rolled loop: this code runs once per CTA
-  // from a cold instruction cache, and every instruction line of an unrolled version costs a fetch.
-  float* obuf = s_inv + kRowsPerBlock;  // [64 rows][kORow floats]
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
-    float4* dst = reinterpret_cast<float4*>(obuf + row * kORow + piece * 8);
-    dst[0] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-    dst[1] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
-  }
-  __syncwarp();  // a thread reads back only what it wrote
-#pragma unroll 1
-  for (int i = 0; i < 8; ++i) {
-    const int idx = i * 128 + (int)threadIdx.x, row = idx >> 4, piece = idx & 15;
-    const int jj = rb * kRowsPerBlock + row;
-    if (jj >= p.T) continue;
-    const float inv = s_inv[row];
-    const float4 a = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8);
-    const float4 b = *reinterpret_cast<const float4*>(obuf + row * kORow + piece * 8 + 4);
-    const float v8[8] = {a.x * inv, a.y * inv, a.z * inv, a.w * inv, b.x * inv, b.y * inv, b.z * inv, b.w * inv};
-    store8(p, r * p.T + jj, head * kD + piece * 8, p.Hq * kD, v8);
-  }
+  // nobody leaves while a CTA of the cluster may still read its shared memory
+  ptx::cluster_arrive();
+  ptx::cluster_wait();
 }
 
 }  // namespace
@@ -584,28 +584,26 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   a.Hq = sh.Hq;
   a.Hkv = sh.Hkv;
   a.n_rb = cascade_detail::ceil_div(T, kRowsPerBlock);
-  a.t_pad = (int)cascade_detail::align_up(sh.T_max, 64);
   a.prefix_cap = prefix_cap;
   a.prefix_len = prefix_len;
   a.anc = tree->d_anc;
   a.out = out;
   a.out_as_operand = out_as_operand ? 1 : 0;
   a.out_lay = operand_layout(R * T, sh.Hq * kD);
-  a.part_o = ctx->attn_part_o;
-  a.part_ml = ctx->attn_part_ml;
   a.c = scale * 1.4426950408889634f;
   a.err = ctx->dev_error;
   a.wait_ns = ctx->wait_limit_ns;
-  a.unit_done = ctx->attn_unit_done;
-  // KV splits: as many as fit on the SMs at once, never more splits than tiles or than the scratch holds
-  const int n_tiles = cascade_detail::ceil_div(prefix_cap, kTileKeys) + cascade_detail::ceil_div(T, kTileKeys);
+  // KV splits (1, 2 or 4 CTAs in a cluster per unit): as many as fit on the SMs at once, each keeping a minimum of
+  // tiles of the longest possible row
+  const int items = cascade_detail::ceil_div(prefix_cap, kTileKeys) + 1;  // prefix tiles + the tree's own tiles as one
   const int units = R * sh.Hq * a.n_rb;
-  int splits = ctx->sm_count / units;
-  if (splits > n_tiles) splits = n_tiles;
-  if (splits > ctx->attn_max_splits) splits = ctx->attn_max_splits;
-  // merging splits costs a few microseconds of its own: not worth it for a handful of tiles
-  if (splits > 1 && n_tiles - cascade_detail::ceil_div(n_tiles, splits) < 4) splits = 1;
-  if (splits < 1) splits = 1;
+  int splits = 1;
+  for (int cand = kMaxSplits; cand > 1; cand /= 2) {
+    if (units * cand <= ctx->sm_count && cascade_detail::ceil_div(items, cand) >= ctx->attn_min_tiles_per_split) {
+      splits = cand;
+      break;
+    }
+  }
   a.splits = splits;
 
   const uint64_t dq[4] = {(uint64_t)kD, (uint64_t)sh.Hq, (uint64_t)T, (uint64_t)R};
@@ -631,11 +629,21 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_tree_attn_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     configured = true;
   }
-  dim3 grid(splits, sh.Hq * a.n_rb, R);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(splits, sh.Hq * a.n_rb, R);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;  // the splits of one (row, head, row block) are one cluster
+  attr[0].val.clusterDim.x = splits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   {
     KernelScope ks(ctx, K_TREE_ATTN, s);
-    k_tree_attn_bf16<<<grid, kThreads, kSmemBytes, s>>>(*mq, *mkp, *mvp, *mkt, *mvt, a);
+    CASCADE_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_tree_attn_bf16, *mq, *mkp, *mvp, *mkt, *mvt, a));
   }
-  CASCADE_CUDA_TRY(cudaGetLastError());
   return CASCADE_OK;
 }

@@ -70,11 +70,8 @@ struct cascade_ctx {
   float* gemm_scratch = nullptr;         // tensor-core GEMM: partial accumulators of tiles split between CTAs
   unsigned int* gemm_flags = nullptr;    // one hand-off flag per CTA (zero between launches)
 
-  // tree attention, split-KV partial results
-  int attn_max_splits = 1;
-  float* attn_part_o = nullptr;   // [R*Hq*splits][T_pad][D]
-  float2* attn_part_ml = nullptr;  // [R*Hq*splits][T_pad]  (row max, row sum)
-  unsigned int* attn_unit_done = nullptr;  // [R*Hq*row blocks] finished-split counters (zero between launches)
+  // tree attention: a KV split must keep at least this many 128-key tiles (merging splits has a fixed cost)
+  int attn_min_tiles_per_split = 2;
 
   // LM head
   int head_m_pad = 0;             // B*T_max rounded up to 128

@@ -64,6 +64,55 @@ def test_full_width_step_through_one_layer(name):
     wl.close()
 
 
+def test_two_full_width_layers_each_against_the_checker_on_the_same_input():
+    """The decode loop's widths (hidden 4096, 32 heads x 128, SwiGLU 11008, vocabulary 16384, a 64-row prompt cache,
+    61 tree rows), two layers.  Layer 1 is compared with the checker from the token embeddings; layer 2 and the head
+    are compared with the checker run on the DEVICE's layer-1 output, so that both sides round the same values to
+    bf16 where the workload stores bf16 (rotated queries, keys, values).  End to end -- the checker on its own
+    layer-1 output -- the two computations part by isolated bf16 steps in layer 2's operands; that figure is
+    reported and held to twice the single-layer tolerance."""
+    w = synth.workload("janus", prefix_len=64)
+    parent = w.parent()
+    host = synth.layer_step_inputs(w, np.random.default_rng(w.seed), parent, 2)
+    first = dict(host, layers=host["layers"][:1], k_prefix=host["k_prefix"][:1], v_prefix=host["v_prefix"][:1])
+    wl1 = LayerWorkload(w, n_layers=1, host=first)
+    s1 = wl1.run(0)
+    torch.cuda.synchronize()
+    wl1.ctx.check()
+    x1_dev = s1.out["hidden_out"].cpu().numpy().astype(np.float64)
+    wl1.close()
+    wl2 = LayerWorkload(w, n_layers=2, keep_logits=True, host=host)
+    s2 = wl2.run(0)
+    torch.cuda.synchronize()
+    wl2.ctx.check()
+    x2_dev = s2.out["hidden_out"].cpu().numpy()
+    logits = s2.out["logits"].cpu().numpy()
+    # layer 1 from the embeddings
+    x0 = np.asarray(host["embed"], np.float64)[np.concatenate([host["tok"], host["tok"]], 0)]
+    x1_ref, *_ = O.decoder_layer(x0, host["layers"][0], host["k_prefix"][0], host["v_prefix"][0], host["prefix_len"], parent,
+                                 w.n_heads, w.head_dim, w.eps, w.rope_base, True)
+    e1 = np.abs(x1_dev - x1_ref).max()
+    assert e1 < HIDDEN_TOL, e1
+    # layer 2 + head from the device's layer-1 output
+    x2_ref, q, k, v = O.decoder_layer(x1_dev, host["layers"][1], host["k_prefix"][1], host["v_prefix"][1], host["prefix_len"],
+                                      parent, w.n_heads, w.head_dim, w.eps, w.rope_base, True)
+    e2 = np.abs(x2_dev - x2_ref).max()
+    assert e2 < HIDDEN_TOL, e2
+    assert np.abs(s2.out["k_tree_out"][1].float().cpu().numpy() - k).max() < 4e-2
+    head = O.lm_head_cfg(x2_ref, host["gamma_final"], w.eps, host["w_head"], w.cfg_scale, 1.0)
+    e_logits = np.abs(logits - head["logits"]).max()
+    assert e_logits < LOGIT_TOL, e_logits
+    # end to end, for the record
+    x2_own, *_ = O.decoder_layer(x1_ref, host["layers"][1], host["k_prefix"][1], host["v_prefix"][1], host["prefix_len"], parent,
+                                 w.n_heads, w.head_dim, w.eps, w.rope_base, True)
+    own = O.lm_head_cfg(x2_own, host["gamma_final"], w.eps, host["w_head"], w.cfg_scale, 1.0)
+    e_end = np.abs(logits - own["logits"]).max()
+    assert e_end < 2 * LOGIT_TOL, e_end
+    print(f"two full-width layers: hidden after layer 1 {e1:.2e}, after layer 2 (same input) {e2:.2e}, logits (same input) "
+          f"{e_logits:.2e}, logits end to end {e_end:.2e}")
+    wl2.close()
+
+
 @pytest.mark.parametrize("B", [1, 2])
 def test_head_at_vocabulary_65536(B):
     """61 and 122 activation rows against a [65536, 4096] head: 512 vocabulary tiles x 32 K blocks over 148 CTAs, so

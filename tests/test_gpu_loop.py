@@ -19,6 +19,9 @@ pytestmark = pytest.mark.gpu
     ("mini", dict(B=2, tree="topk32", prefix_len=40), 2, 3, None),
     ("mini", dict(B=1, tree="topk60", prefix_len=130), 3, 2, None),
     ("mini", dict(B=2, tree="topk32", prefix_len=40), 2, 4, 1),     # steps after the first replay a recorded CUDA graph
+    # the decode loop's own widths (hidden 4096, 32 heads x 128, SwiGLU 11008, vocabulary 16384, 64-row prompt cache,
+    # 61-row trees): two of its layers, two steps, the second replayed from a recorded graph
+    pytest.param("janus", dict(prefix_len=64), 2, 2, 1, id="full-width-2-layers"),
 ])
 def test_decode_loop(name, over, n_layers, steps, graph_after):
     w = synth.workload(name, **over)
@@ -41,7 +44,12 @@ def test_decode_loop(name, over, n_layers, steps, graph_after):
         torch.cuda.synchronize()
         o = loop.set.out
         logits = o["logits"].cpu().numpy()
-        assert np.abs(logits - ref["head"]["logits"]).max() < 3e-2
+        # 3e-2 per step through one layer.  At full width the second layer rounds its queries, keys and values to
+        # bf16 from inputs that already differ from the checker's in the last bits, so isolated elements land on the
+        # neighbouring bf16 value (a 0.4 % step) in one computation and not in the other: the two part by up to one
+        # layer's tolerance per layer.  (tests/test_gpu_fullsize.py holds every layer to 3e-2 on identical inputs.)
+        tol = 3e-2 * (n_layers if name != "mini" else 1)
+        assert np.abs(logits - ref["head"]["logits"]).max() < tol
         feat = o["feat"].cpu().numpy().astype(np.float64)
         rows = [O.relaxed_accept(feat[b], logits[b], tok[b], parent, p[b], u[b], w.tau_pos, w.tau_seq, w.tvd_budget)
                 for b in range(B)]
