@@ -62,7 +62,7 @@ struct cascade_ctx {
   bool timing = false;
   unsigned long long wait_limit_ns = 2000000000ull;  // limit of every bounded device-side wait (cascade_set_wait_limit)
   // cudaFuncSetAttribute is per device and a context is bound to one device: what has been set is kept here
-  int gemm_smem_configured[3] = {0, 0, 0};
+  int gemm_smem_configured[6] = {0, 0, 0, 0, 0, 0};
   bool attn_configured = false, filter_configured = false;
   std::vector<TimedLaunch> timed;        // event pairs recorded since the last read
   std::vector<cudaEvent_t> event_pool;   // spare events

@@ -43,6 +43,7 @@
 namespace {
 
 constexpr int kThreads = 192;       // warp 0: TMA, warp 1: UMMA issue + TMEM alloc, warps 2-5: epilogue
+constexpr int kLeanThreads = 320;   // ... warps 2-9: epilogue of the sliced projections
 constexpr int kTileN = 128;         // weight rows per accumulator (UMMA M)
 constexpr int kSpan = 64;           // K elements per stage (one 128-byte swizzle span)
 constexpr int kMaxStages = 8;
@@ -138,8 +139,14 @@ struct SegmentWalk {
 };
 
 // kHalves: accumulators (128 weight rows each) per work tile.  kSpans: 64-wide K spans per stage.
-template <int kHalves, int kSpans>
-__global__ void __launch_bounds__(kThreads, 1)
+// kLean: the plain-store epilogue of the sliced projections, run by EIGHT warps (two per TMEM lane quadrant, each
+// group of four taking every other 32-column block of the tile).  What a CTA does after its last UMMA is not hidden
+// behind anything, and all CTAs get there together: four warps drain a 128 KB tile at about 30 GB/s per SM (their
+// instruction stream, not the memory system, sets that rate), eight in half the time.  The general epilogue
+// (softmax partials, candidate gather, split-tile hand-off) needs more registers than 320 threads leave and keeps
+// its four warps.
+template <int kHalves, int kSpans, bool kLean>
+__global__ void __launch_bounds__(kLean ? kLeanThreads : kThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
   constexpr int kWSpanBytes = kHalves * kTileWBytes;  // weights of one span
   constexpr int kWBytes = kSpans * kWSpanBytes;       // weights of one stage: span after span
@@ -147,9 +154,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
   __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], tmem_full[2], tmem_empty[2];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ __align__(16) float st[kStCols * kStRow];
-  __shared__ int s_gather_n;
-  __shared__ int4 s_gather[kGatherCap];  // {weight row in tile, parent column, grandparent column, idx}
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -164,7 +168,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
     }
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&tmem_full[i], 1);
-      ptx::mbar_init(&tmem_empty[i], 128);
+      ptx::mbar_init(&tmem_empty[i], kLean ? kLeanThreads - 64 : 128);
     }
     s_abort = 0;
     ptx::fence_mbar_init();
@@ -281,8 +285,73 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const GemmArgs p) {
         ptx::umma_commit(&tmem_full[acc]);
       }
     }
+  } else if constexpr (kLean) {
+    // ---------------- plain-store epilogue (256 threads: two groups of four warps) ----------------
+    __shared__ __align__(16) float st2[2][32 * kTileN];   // per group: 32 activation rows x 128 weight rows
+    const int quad = warp & 3;                  // TMEM lane quadrant this warp may read
+    const int vl = quad * 32 + lane;            // weight row within the tile
+    const int group = (warp - 2) >> 2, gwarp = (warp - 2) & 3;
+    float* const stg = st2[group];
+    const GemmEpilogue& e = p.epi;
+    const int NB = p.NB;
+    const int blocks_per_half = (NB + 31) / 32;
+    uint32_t seg_i = 0;
+    SegmentWalk walk(p);
+    Segment sg;
+    while (walk.next(sg)) {
+      const uint32_t acc = seg_i & 1u, aph = (seg_i >> 1) & 1u;
+      ++seg_i;
+      const int macro = sg.tile / p.n_mchunks, m0 = (sg.tile % p.n_mchunks) * NB;
+      float* const c_out = e.C + (size_t)sg.slice * p.slice_stride;
+      if (!ptx::mbar_wait(&tmem_full[acc], aph, abort_flag, p.err, p.wait_ns)) break;
+      ptx::tc_fence_after();
+#pragma unroll 1  // run-once code at the end of the kernel: one copy of the block's instructions
+      for (int blk = group; blk < kHalves * blocks_per_half; blk += 2) {
+        const int half = blk / blocks_per_half, c0 = (blk - half * blocks_per_half) * 32;
+        const int n_tile = macro * kHalves + half;
+        if (n_tile * kTileN >= p.N) break;      // second half of the last work tile lies beyond N
+        const int n_cols = min(32, NB - c0);
+        const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * (uint32_t)p.acc_cols +
+                                half * (uint32_t)NB + (uint32_t)c0;
+        float v[32];
+        if (n_cols == 32) {
+          ptx::tmem_ld32(t_addr, v);
+        } else {
+          ptx::tmem_ld16(t_addr, v);            // NB is a multiple of 16: the last block of a half may hold 16 columns
+        }
+        ptx::named_bar_sync(1 + group, 128);    // the previous block has been read out of the staging buffer
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (i < n_cols) stg[i * kTileN + vl] = v[i];
+        ptx::named_bar_sync(1 + group, 128);
+        // output rows are contiguous over the weight rows: a warp writes the 128 weight rows of an activation row
+        // with one 16-byte store per lane
+        const int row0 = m0 + c0, n0 = n_tile * kTileN + 4 * lane;
+        const bool wide = (e.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(c_out) & 15u) == 0 && n0 + 4 <= p.N;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int i = gwarp + 4 * k;
+          if (i >= n_cols || row0 + i >= p.M) continue;
+          const float4 x = *reinterpret_cast<const float4*>(stg + i * kTileN + 4 * lane);
+          float* dst = c_out + (size_t)(row0 + i) * e.ldc + n0;
+          if (wide) {
+            *reinterpret_cast<float4*>(dst) = x;
+          } else {
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              if (n0 + q < p.N) dst[q] = xs[q];
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&tmem_empty[acc]);
+    }
   } else {
     // ---------------- epilogue (128 threads) ----------------
+    __shared__ __align__(16) float st[kStCols * kStRow];
+    __shared__ int s_gather_n;
+    __shared__ int4 s_gather[kGatherCap];  // {weight row in tile, parent column, grandparent column, idx}
     const int quad = warp & 3;                  // TMEM lane quadrant this warp may read
     const int vl = quad * 32 + lane;            // weight row within the tile
     const int eid = (warp - 2) * 32 + lane;     // 0..127
@@ -643,7 +712,9 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   // (With at most 64 activation rows, 256-row tiles measured no faster on the stream and split the LM
   // head of a 16384-token vocabulary over too few tiles.)
   const int halves = pick_halves(a.NB, epi.splits > 0);
-  const int budget = 227 * 1024 - 20 * 1024 - 1024;  // static shared + alignment slack
+  // static shared memory (general epilogue: 19 KB; eight-warp epilogue: two 16 KB staging buffers) + alignment slack
+  const bool lean_cfg = epi.splits >= 1 && epi.part == nullptr && !epi.accumulate && epi.C != nullptr && epi.tok == nullptr;
+  const int budget = 227 * 1024 - (lean_cfg ? 33 : 20) * 1024 - 1024;
   const int span_bytes = halves * kTileWBytes + 2 * a.NB * kSpan * 2;
   const int spans = (K % (2 * kSpan) == 0 && budget / (2 * span_bytes) >= 3) ? 2 : 1;
   const int stage_bytes = spans * span_bytes;
@@ -671,9 +742,12 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   if (tw == nullptr) return CASCADE_ERR_CUDA;
   const int smem = a.stages * stage_bytes + 1024;
   if (halves == 2 && spans == 2) return CASCADE_ERR_UNSUPPORTED_SHAPE;  // cannot happen: such stages do not fit
-  auto kern = halves == 2 ? k_gemm_tc<2, 1> : (spans == 2 ? k_gemm_tc<1, 2> : k_gemm_tc<1, 1>);
+  // the sliced projections (plain store of every piece into its own matrix) take the eight-warp epilogue
+  const bool lean = epi.splits >= 1 && epi.part == nullptr && !epi.accumulate && epi.C != nullptr && epi.tok == nullptr;
+  auto kern = lean ? (halves == 2 ? k_gemm_tc<2, 1, true> : (spans == 2 ? k_gemm_tc<1, 2, true> : k_gemm_tc<1, 1, true>))
+                   : (halves == 2 ? k_gemm_tc<2, 1, false> : (spans == 2 ? k_gemm_tc<1, 2, false> : k_gemm_tc<1, 1, false>));
   int* configured_smem = ctx->gemm_smem_configured;
-  const int kern_i = halves == 2 ? 2 : spans - 1;
+  const int kern_i = (halves == 2 ? 2 : spans - 1) + (lean ? 3 : 0);
   if (smem > configured_smem[kern_i]) {
     CASCADE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     configured_smem[kern_i] = smem;
@@ -687,7 +761,7 @@ int launch_gemm_tc(cascade_ctx* ctx, const __nv_bfloat16* W, int N, int K, const
   a.unit_r = (int)(a.units % grid);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(lean ? kLeanThreads : kThreads);
   cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
