@@ -398,6 +398,22 @@ int cascade_kv_append(cascade_ctx* ctx, const cascade_tree* tree, int32_t n_laye
 int cascade_filter_logits(cascade_ctx* ctx, float* logits, int32_t n_rows, int32_t top_k, float top_p,
                           int32_t* kept_count, void* stream);
 
+/* ---- the drafter's training loss (outside the verification step) ---------------------------------- */
+/* Section 4.3, Eq. 4: the soft cross-entropy between the target distribution and the drafter's at every position k
+ * of a target-generated sequence, weighted by c (2 in the paper's experiments, Appendix D.1) where the target's
+ * hidden states of positions k and k+1 satisfy the convergence criterion of Eq. 2 (cosine >= tau_seq), by 1 elsewhere
+ * and at the last position:
+ *     loss_out[k] = - w_k * sum_v softmax(target_logits[k])[v] * log softmax(draft_logits[k])[v]
+ *   target_logits, draft_logits [K,V] float; feat [K,h] float (target hidden states); DEVICE pointers.
+ *   loss_out [K] float; weight_out [K] float or NULL (w_k); total_out [1] float or NULL (sum of loss_out, added in
+ *   index order).  No context is needed and nothing is allocated; two kernels on `stream`.
+ * Only the forward value is computed (the gradient with respect to draft_logits[k] is w_k (p_k - q_k), which a
+ * training framework forms from its own softmax).  Errors: CASCADE_ERR_INVALID_ARG (null pointers, sizes < 1,
+ * c <= 0, NaN threshold). */
+int cascade_drafter_loss(const float* target_logits, const float* draft_logits, const float* feat, int32_t K, int32_t V,
+                         int32_t h, float tau_seq, float c, float* loss_out, float* weight_out, float* total_out,
+                         void* stream);
+
 /* ---- acceptance without any device allocation --------------------------------------------------- */
 /* The paper has no counterpart to this entry point; it exists for deployment.  Some callers of this
  * library may not allocate device memory at all: a plug-in running inside a serving process that

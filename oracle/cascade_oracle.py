@@ -17,7 +17,8 @@ Parity pins (tests/test_oracle_*.py): every function below is pinned to somethin
 textbook causal / decode attention, CFG end points and linearity, closed-form cosine cases, reduction
 to Algorithm 1 with the relaxation off, an independently written sequential walk of Algorithm 2,
 brute-force path enumeration, threshold monotonicity with an unbounded budget, hand-computed trees,
-exact recovery of the target distribution by accept test + residual draw (Algorithm 1's guarantee),
+exact recovery of the target distribution by accept test + residual draw (Algorithm 1's guarantee), the
+library's soft cross-entropy / KL divergence + entropy for the drafter loss of Eq. 4,
 the library's top-k and a brute-force nucleus for the truncation of the target distribution.
 `decoder_layer` (architecture from the workload definition, not from the paper) is pinned against an
 ordinary causal block built from torch's library routines: on a chain with an empty prefix, and on a
@@ -397,6 +398,26 @@ def residual_token(logits_row, draft_row, any_rejected, u):
     c = np.cumsum(w)
     v = int(np.searchsorted(c, float(u) * c[-1], side="right"))
     return min(v, len(w) - 1), total
+
+
+def drafter_loss(target_logits, draft_logits, feat, tau_seq, c):
+    """The drafter's training loss of Section 4.3, Eq. 4: a soft cross-entropy between the target distribution q_k
+    and the drafter's distribution p_k at every position k of a target-generated sequence,
+        L = - sum_k w_k sum_v q_k(v) log p_k(v),
+    re-weighted where consecutive target predictions converge: w_k = c if the pair (k, k+1) satisfies the
+    convergence criterion of Eq. 2, cos(F_k, F_{k+1}) >= tau_seq on the target's hidden states, else 1 (the last
+    position has no successor: w = 1).  target_logits, draft_logits [K,V]; feat [K,h].
+    Returns (per-position weighted loss [K], weights [K], total)."""
+    q = softmax(np.asarray(target_logits, np.float64))
+    lp = np.asarray(draft_logits, np.float64)
+    log_p = lp - log_sum_exp(lp)[..., None]
+    K = q.shape[0]
+    ce = -(q * log_p).sum(-1)
+    w = np.ones(K)
+    for k in range(K - 1):
+        if cosine(feat[k], feat[k + 1]) >= tau_seq:
+            w[k] = c
+    return w * ce, w, float((w * ce).sum())
 
 
 def filter_logits(logits, top_k, top_p):

@@ -30,7 +30,7 @@ EXPORTS = [
     "cascade_similarity", "cascade_relaxed_accept", "cascade_select_path", "cascade_verify_step",
     "cascade_verify_step_host", "cascade_accept_static", "cascade_bonus_token", "cascade_kv_append",
     "cascade_filter_logits", "cascade_set_wait_limit", "cascade_wait_probe",
-    "cascade_tree_update_device", "cascade_tree_download",
+    "cascade_tree_update_device", "cascade_tree_download", "cascade_drafter_loss",
 ]
 
 
@@ -109,6 +109,7 @@ def lib() -> C.CDLL:
         L.cascade_filter_logits.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_float, vp, vp]
         L.cascade_tree_update_device.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, vp, vp]
         L.cascade_tree_download.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.cascade_drafter_loss.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_float, vp, vp, vp, vp]
         L.cascade_set_wait_limit.argtypes = [vp, C.c_int64]
         L.cascade_wait_probe.argtypes = [vp, vp, vp]
         _lib = L
@@ -353,3 +354,11 @@ def cascade_kv_append(ctx, tree, step: Step, k_tree, v_tree, path_nodes, path_le
     """Appends the accepted path's rows to the caches named in `step.layers` (a Step made by make_step)."""
     _check(lib().cascade_kv_append(ctx.handle, tree.handle, step.n_layers, step.layers, _ptr(k_tree), _ptr(v_tree),
                                    _ptr(path_nodes), _ptr(path_len), prefix_cap, _ptr(prefix_len), _stream()))
+
+
+def cascade_drafter_loss(target_logits, draft_logits, feat, tau_seq, c, loss_out, weight_out=None, total_out=None):
+    """Eq. 4 of the paper on [K,V] target / drafter logits and [K,h] target hidden states (device tensors)."""
+    K, V = target_logits.shape
+    _check(lib().cascade_drafter_loss(_ptr(target_logits), _ptr(draft_logits), _ptr(feat), K, V, feat.shape[-1],
+                                      float(tau_seq), float(c), _ptr(loss_out), _ptr(weight_out), _ptr(total_out),
+                                      _stream()))

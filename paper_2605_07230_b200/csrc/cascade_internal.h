@@ -71,7 +71,7 @@ struct cascade_ctx {
   unsigned int* gemm_flags = nullptr;    // one hand-off flag per CTA (zero between launches)
 
   // tree attention: a KV split must keep at least this many 128-key tiles (merging splits has a fixed cost)
-  int attn_min_tiles_per_split = 2;
+  int attn_min_tiles_per_split = 3;
 
   // LM head
   int head_m_pad = 0;             // B*T_max rounded up to 128

@@ -186,6 +186,12 @@ int launch_head_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv_bflo
     e.cand_parent = cand_parent;
     e.cand_gparent = cand_gparent;
   }
+  // With more than 128 activation rows (several row chunks) the head is no longer a weight stream: every weight tile
+  // is used once per chunk, there are hundreds of (tile, chunk) items, and what bounds a 128 x 128 item is the
+  // shared-memory fill per UMMA (16 KB of weights + 32 KB of activation pair for eight instructions).  Whole
+  // items of 256 weight rows (two accumulators on one activation stage, nothing cut along K, no hand-off) double
+  // the tensor work per byte taken in.
+  if (operand_layout(sh.B * tree->T, sh.h).n_chunks > 1) e.splits = 1;
   return launch_gemm_tc(ctx, w_head, sh.V, sh.h, ctx->head_a, sh.B * tree->T, e, K_GEMM_HEAD, s);
 }
 

@@ -303,6 +303,12 @@ def workload(name: str, **over) -> Workload:
                        seed=2),
         "sweep": dict(dtype="bf16", B=8, h=4096, n_heads=32, head_dim=128, V=16384, n_clusters=256, sigma=0.1,
                       prefix_len=1024, tree="topk64", cfg_scale=5.0, tau_pos=0.85, tau_seq=0.5, ffn=11008, seed=3),
+        # LlamaGen-XL-Stage2, the model behind the paper's largest speed-ups.  The paper gives its thresholds, guidance
+        # scale and sequence length (1024 image tokens) but no shape; ASSUMED here: width 1280, SwiGLU 3584, vocabulary
+        # 16384, a 120-token text prefix (that model's published configuration), with its 20 heads of 64 regrouped as
+        # 10 heads of 128 (the bf16 attention kernel takes head size 128), half-way through an image (120 + 512 keys)
+        "llamagen": dict(dtype="bf16", B=1, h=1280, n_heads=10, head_dim=128, V=16384, n_clusters=256, sigma=0.1,
+                         prefix_len=632, tree="topk60", cfg_scale=3.0, tau_pos=0.85, tau_seq=0.5, ffn=3584, seed=5),
         # reduced-width stand-ins of the same structure for CPU-side and quick GPU tests
         "mini": dict(dtype="bf16", B=2, h=512, n_heads=4, head_dim=128, V=2048, n_clusters=64, sigma=0.1,
                      prefix_len=200, tree="topk32", cfg_scale=5.0, tau_pos=0.85, tau_seq=0.5, ffn=1408, seed=4),

@@ -22,7 +22,7 @@ pytestmark = pytest.mark.gpu
 HIDDEN_TOL = 2e-2
 
 
-@pytest.mark.parametrize("name", ["janus", "lumina"])
+@pytest.mark.parametrize("name", ["janus", "lumina", "llamagen"])
 def test_full_width_step_through_one_layer(name):
     w = synth.workload(name)
     wl = LayerWorkload(w, n_layers=1, keep_logits=True)
