@@ -96,3 +96,41 @@ def test_static_scratch_entry_rejects_sizes_beyond_its_array():
     too_many_rows = L.cascade_accept_static(1, 300, big, p, 4, None, p, p, p, p, p, p, C.byref(params), 0, p, None,
                                             None, None, p, p, None, None)
     assert too_many_rows == cb.ERR_UNSUPPORTED_SHAPE
+
+
+def test_static_scratch_entry_against_the_checker():
+    """The same entry against the fp64 checker directly: logits are made on the host, the row statistics and
+    candidate logits the entry takes are derived from them with the checker's own helpers, and the decisions must
+    equal the checker's rule on those logits and features (near-threshold nodes set aside as everywhere)."""
+    from oracle import cascade_oracle as O
+    w = synth.workload("mini", B=3, tree="topk32", V=512)
+    parent = w.parent()
+    T = len(parent)
+    rng = np.random.default_rng(77)
+    tok, p = synth.cluster_drafter(rng, parent, w.B, w.V, w.n_clusters)
+    E = synth.clustered_codebook(rng, w.V, w.h, w.n_clusters, w.sigma)
+    feat = (E[tok] + 0.003 * rng.standard_normal((w.B, T, w.h), dtype=np.float32)).astype(np.float32)
+    # target logits that favour each row's own cluster, so that drafted tokens carry real mass
+    logits = (rng.normal(0, 1, (w.B, T, w.V)) + 4.0 * ((np.arange(w.V)[None, None, :] % w.n_clusters) ==
+                                                        (tok[:, :, None] % w.n_clusters))).astype(np.float32)
+    u = synth.uniforms(rng, w.B, T)
+    lse = O.log_sum_exp(logits).astype(np.float32)
+    cp, cg = (x.astype(np.float32) for x in O.candidate_logits(logits, tok, parent))
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(G.DEV)
+    params = cb.Params(w.tau_pos, w.tau_seq, w.tvd_budget, cb.USE_I | cb.USE_C)
+    depth = int(O.tree_depth(parent).max())
+    got = _outputs(w.B, T, depth)
+    cb.cascade_accept_static(w.B, parent, dev(feat), w.h, None, dev(lse), dev(cp), dev(cg), dev(tok), dev(p), dev(u), params,
+                             cb.SELECT_LONGEST, got["accept"], got["q_relaxed"], got["tvd_out"], got["near"], got["nodes"],
+                             got["plen"], got["tvd_used"])
+    torch.cuda.synchronize()
+    rows = [O.relaxed_accept(feat[b].astype(np.float64), logits[b], tok[b], parent, p[b], u[b], w.tau_pos, w.tau_seq,
+                             w.tvd_budget) for b in range(w.B)]
+    st = G.compare_decisions(parent, rows, got["accept"].cpu().numpy(), got["nodes"].cpu().numpy(),
+                             got["plen"].cpu().numpy(), cb.SELECT_LONGEST)
+    assert st["nodes_compared"] > 0.8 * st["nodes"]
+    qR = got["q_relaxed"].cpu().numpy()
+    for b in range(w.B):
+        if not rows[b]["near"].any():
+            assert np.abs(qR[b] - rows[b]["q_relaxed"]).max() < 1e-4
+    assert sum(int(r["accept"].sum()) for r in rows) > w.B     # drafts were accepted
