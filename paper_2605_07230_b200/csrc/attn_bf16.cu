@@ -40,17 +40,20 @@ namespace {
 
 constexpr int kD = 128;
 constexpr int kTileKeys = 128;
-constexpr int kRowsPerBlock = 64;
+constexpr int kRowsNarrow = 64;   // rows per block with the duplicated Q tile (trees of up to 64 rows)
+constexpr int kRowsWide = 128;    // rows per block without duplication (larger trees)
 constexpr int kSoftmaxThreads = 256;  // warps 0-7
 constexpr int kThreads = 320;         // + warp 8: TMA, warp 9: UMMA issue + TMEM alloc
 constexpr int kQBytes = 128 * kD * 2;        // 32 KB: two 64-wide halves of [128 rows][64] bf16
 constexpr int kPBytes = 128 * kTileKeys * 2;  // 32 KB
 constexpr int kKVTileBytes = kTileKeys * kD * 2;  // 32 KB for K, same for V
 constexpr int kKSlots = 2;     // K tiles in shared memory (a slot is free again once S = Q K^T has read it)
-constexpr int kVSlots = 3;     // V tiles in shared memory (free once O += P V has read it)
+constexpr int kVSlotsNarrow = 3, kVSlotsWide = 2;  // V tiles in shared memory (free once O += P V has read it); the
+                               // wide form holds two P tiles (values and remainders) and has room for two
 constexpr int kPrefetch = 0;   // with a ring of n slots, tile i + n - 1 + kPrefetch is requested into the L2 when tile i is
                                // loaded (measured 0..3 on 20-tile rows: deeper requests delay the loads that are waited for)
-constexpr int kSmemBytes = kQBytes + kPBytes + (kKSlots + kVSlots) * kKVTileBytes + 1024;
+constexpr int kSmemBytes = kQBytes + kPBytes + (kKSlots + kVSlotsNarrow) * kKVTileBytes + 1024;
+static_assert(kQBytes + 2 * kPBytes + (kKSlots + kVSlotsWide) * kKVTileBytes + 1024 == kSmemBytes, "both forms use the same shared memory");
 constexpr int kXRow = 132;     // floats per row of the partial-result buffer: 128 outputs, reference, sum, 2 pad
 constexpr int kMaxSplits = 4;
 constexpr float kLazy = 8.f;   // the reference is raised when a score exceeds it by more than this (log2 units)
@@ -93,10 +96,18 @@ __device__ __forceinline__ int float_key(float f) {
 }
 __device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff); }
 
+// kWide = false: row blocks of 64 tree rows, Q tile loaded twice, four threads per row, one P tile whose rows 0-63 /
+// 64-127 hold the values / the remainders (one output product per key tile).  kWide = true (trees of more than 64
+// rows): row blocks of 128, two threads per row with 64 keys each, two P tiles and two output products per key tile
+// into the same accumulator -- one pass over the keys for up to 128 rows instead of one per 64.
+template <bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
 k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kp,
                  const __grid_constant__ CUtensorMap tm_vp, const __grid_constant__ CUtensorMap tm_kt,
                  const __grid_constant__ CUtensorMap tm_vt, const AttnArgs p) {
+  constexpr int kRowsPerBlock = kWide ? kRowsWide : kRowsNarrow;
+  constexpr int kVSlots = kWide ? kVSlotsWide : kVSlotsNarrow;
+  constexpr int kKeysPerThread = kWide ? 64 : 32;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t q_full, k_full[kKSlots], k_empty[kKSlots], v_full[kVSlots], v_empty[kVSlots],
       s_full[2], s_empty[2], p_full, o_full, ref_ready, peers_ready;
@@ -107,7 +118,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-  const uint32_t q_addr = smem_base, p_addr = smem_base + kQBytes, k_ring = p_addr + kPBytes,
+  const uint32_t q_addr = smem_base, p_addr = smem_base + kQBytes, k_ring = p_addr + (kWide ? 2 : 1) * kPBytes,
                  v_ring = k_ring + kKSlots * kKVTileBytes;
 
   if (threadIdx.x == kSoftmaxThreads) {  // the TMA warp's first loads should not wait for their descriptors
@@ -153,7 +164,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     s_abort = 0;
     ptx::fence_mbar_init();
   }
-  if (threadIdx.x < 3 * kRowsPerBlock) (&s_rowmax[0][0])[threadIdx.x] = float_key(-INFINITY);
+  for (int i = threadIdx.x; i < 3 * kRowsPerBlock; i += kThreads) (&s_rowmax[0][0])[i] = float_key(-INFINITY);
   __syncthreads();  // barriers are initialised: the producers start streaming at once
   ptx::cluster_arrive();  // ... and the other CTAs of the cluster may signal this one once they have seen this
   volatile int* abort_flag = &s_abort;
@@ -168,9 +179,10 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   const uint32_t tmem_base = warp != 8 ? s_tmem_base : 0u;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 256;
-  float* xbuf = reinterpret_cast<float*>(smem + kQBytes + kPBytes);  // partial result, in the K ring once the loop is over
+  // partial result [rows][kXRow], in the K (and V) ring once the loop is over
+  float* xbuf = reinterpret_cast<float*>(smem + kQBytes + (kWide ? 2 : 1) * kPBytes);
   // small arrays of the end phase, in the Q tile's place (idle once the last scores have been issued)
-  float (*s_lsum)[kRowsPerBlock] = reinterpret_cast<float (*)[kRowsPerBlock]>(smem);          // [4]: a row's four partial sums
+  float (*s_lsum)[kRowsPerBlock] = reinterpret_cast<float (*)[kRowsPerBlock]>(smem);          // a row's four (two) partial sums: 1 KB
   float (*s_w)[kRowsPerBlock] = reinterpret_cast<float (*)[kRowsPerBlock]>(smem + 1024);      // [kMaxSplits]: merge weights
   float* s_inv = reinterpret_cast<float*>(smem + 1024 + kMaxSplits * kRowsPerBlock * 4);
 
@@ -189,7 +201,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int half = 0; half < 2; ++half)
           for (int copy = 0; copy < 2; ++copy)
             ptx::tma_load_4d(smem + half * (kQBytes / 2) + copy * (64 * 128), &tm_q, half * 64, head,
-                             rb * kRowsPerBlock, r, &q_full);
+                             rb * kRowsPerBlock + (kWide ? copy * 64 : 0), r, &q_full);
       }
       int slot = 0;
       uint32_t ph = 0;
@@ -281,6 +293,14 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const uint64_t vd = ptx::umma_desc_sw128_strides(v_addr + ks * 2048, kKVTileBytes / 2, 1024);
             ptx::umma_bf16(tmem_o, pd, vd, idesc_o, (ip | ks) != 0);  // O accumulates across tiles
           }
+          if constexpr (kWide) {   // the remainders' tile into the same accumulator
+#pragma unroll
+            for (int ks = 0; ks < kTileKeys / 16; ++ks) {
+              const uint64_t pd = ptx::umma_desc_sw128(p_addr + kPBytes + (ks >> 2) * (128 * 128) + (ks & 3) * 32);
+              const uint64_t vd = ptx::umma_desc_sw128_strides(v_addr + ks * 2048, kKVTileBytes / 2, 1024);
+              ptx::umma_bf16(tmem_o, pd, vd, idesc_o, 1u);
+            }
+          }
           ptx::umma_commit(&o_full);
           ptx::umma_commit(&v_empty[vs_slot]);
           if (++vs_slot == kVSlots) {
@@ -306,9 +326,11 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
   } else {
     // ---------------- softmax warps ----------------
-    const int quad = warp & 3, sub = warp >> 2;   // TMEM lane quadrant; which 32 of the quadrant's 64 keys
-    const int row = (quad & 1) * 32 + lane;       // tree row within the block; TMEM lanes row and row + 64 belong to it
-    const int kofs = (quad >> 1) * 64 + sub * 32; // first key (within a tile) of this thread's 32
+    const int quad = warp & 3, sub = warp >> 2;   // TMEM lane quadrant; which half of the quadrant's keys
+    // narrow: tree row = lane within half the quadrants, TMEM lanes row and row + 64 belong to it, 32 keys per thread;
+    // wide: tree row = TMEM lane, 64 keys per thread
+    const int row = kWide ? quad * 32 + lane : (quad & 1) * 32 + lane;
+    const int kofs = kWide ? sub * 64 : (quad >> 1) * 64 + sub * 32;  // first key (within a tile) of this thread's share
     const int j = rb * kRowsPerBlock + row;       // tree row
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint64_t anc_w[4] = {0, 0, 0, 0};
@@ -318,8 +340,9 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     // P rows `row` (bf16 value) and `row + 64` (remainder); this thread's 32 keys are 4 pieces of 16 bytes in the
     // 64-key column block (quad >> 1), at piece positions 4 sub .. 4 sub + 3 before the swizzle
-    const uint32_t p_hi_row = p_addr + (quad >> 1) * (128 * 128) + row * 128;
-    const uint32_t p_lo_row = p_hi_row + 64 * 128;
+    // (wide: rows `row` of the value tile and of the remainder tile, all 8 pieces of column block `sub`)
+    const uint32_t p_hi_row = p_addr + (kWide ? sub : (quad >> 1)) * (128 * 128) + row * 128;
+    const uint32_t p_lo_row = p_hi_row + (kWide ? kPBytes : 64 * 128);
     const uint32_t o_cols = tmem_o + lane_addr + sub * 64;  // the 64 output columns this thread rescales / reads
     float m_ref = -INFINITY;   // the row's reference (same value in the row's four threads)
     float l_run = 0.f;         // sum of this thread's weights
@@ -332,30 +355,35 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       const int key0 = (in_prefix ? tile : tile - n_ptiles) * kTileKeys + kofs;
       // visibility of this thread's 32 keys (rows beyond T see the prefix like any other: their query is the
       // zero fill of the tensor map and nothing of theirs is ever stored; that keeps the test below uniform)
-      uint32_t vis;
+      constexpr uint64_t kAll = kWide ? ~0ull : 0xffffffffull;
+      uint64_t vis;
       if (in_prefix) {
         const int nvis = P - key0;
-        vis = nvis <= 0 ? 0u : (nvis >= 32 ? ~0u : ((1u << nvis) - 1u));
+        vis = nvis <= 0 ? 0ull : (nvis >= kKeysPerThread ? kAll : ((1ull << nvis) - 1ull));
       } else {
-        vis = (uint32_t)(anc_w[(key0 >> 6) & 3] >> (key0 & 63));
+        vis = (anc_w[(key0 >> 6) & 3] >> (key0 & 63)) & kAll;
       }
-      float sc[32];
-      ptx::tmem_ld32(tmem_s + lane_addr + (i & 1) * 128 + kofs, sc);
+      float sc[kKeysPerThread];
+      if constexpr (kWide) {
+        ptx::tmem_ld64(tmem_s + lane_addr + (i & 1) * 128 + kofs, sc);
+      } else {
+        ptx::tmem_ld32(tmem_s + lane_addr + (i & 1) * 128 + kofs, sc);
+      }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&s_empty[i & 1]);
       // A tile every row of the warp sees whole (all but the last prefix tile) needs no masking, and with a
       // positive scale the maximum can be taken before scaling: weight = 2^(s * c - ref) in one multiply-add.
-      const bool whole = p.c > 0.f && __all_sync(0xffffffffu, vis == ~0u);
+      const bool whole = p.c > 0.f && __all_sync(0xffffffffu, vis == kAll);
       float m_tile = -INFINITY;
       if (whole) {
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int k = 0; k < 32; ++k) m4[k & 3] = fmaxf(m4[k & 3], sc[k]);
+        for (int k = 0; k < kKeysPerThread; ++k) m4[k & 3] = fmaxf(m4[k & 3], sc[k]);
         m_tile = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * p.c;
       } else {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          sc[k] = ((vis >> k) & 1u) ? sc[k] * p.c : -INFINITY;
+        for (int k = 0; k < kKeysPerThread; ++k) {
+          sc[k] = ((vis >> k) & 1ull) ? sc[k] * p.c : -INFINITY;
           m_tile = fmaxf(m_tile, sc[k]);
         }
       }
@@ -372,7 +400,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
       float rowsum = 0.f;
 #pragma unroll
-      for (int k = 0; k < 32; ++k) {
+      for (int k = 0; k < kKeysPerThread; ++k) {
         sc[k] = ptx::ex2(fmaf(sc[k], mul, -m_use));
         rowsum += sc[k];
       }
@@ -382,7 +410,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // 2^-96 of the result either way.
         rowsum = 0.f;
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
+        for (int k = 0; k < kKeysPerThread; ++k) {
           sc[k] = fminf(sc[k], 1.329228e36f);
           rowsum += sc[k];
         }
@@ -399,7 +427,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (__any_sync(0xffffffffu, alpha != 1.f)) {
           // rare: this tile's weights and what has been accumulated so far move to the new reference
 #pragma unroll
-          for (int k = 0; k < 32; ++k) sc[k] *= alpha;
+          for (int k = 0; k < kKeysPerThread; ++k) sc[k] *= alpha;
           rowsum *= alpha;
           l_run *= alpha;
           ptx::tc_fence_after();
@@ -414,9 +442,9 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           ptx::tc_fence_before();
         }
       }
-      // the bf16 value and what its rounding dropped, four 16-byte pieces each
+      // the bf16 value and what its rounding dropped, four (eight) 16-byte pieces each
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < kKeysPerThread / 8; ++c) {
         uint32_t hi[4], lo[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -424,7 +452,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           hi[k] = ptx::pack_bf16x2(a, b);
           lo[k] = ptx::pack_bf16x2(a - __uint_as_float(hi[k] << 16), b - __uint_as_float(hi[k] & 0xffff0000u));
         }
-        const uint32_t piece = (uint32_t)((4 * sub + c) ^ (row & 7)) << 4;
+        const uint32_t piece = (uint32_t)(((kWide ? 0 : 4 * sub) + c) ^ (row & 7)) << 4;
         ptx::st_shared_v4(p_hi_row + piece, hi[0], hi[1], hi[2], hi[3]);
         ptx::st_shared_v4(p_lo_row + piece, lo[0], lo[1], lo[2], lo[3]);
       }
@@ -439,11 +467,11 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if (ok && n > 0) have_o = ptx::mbar_wait(&o_full, (n - 1) & 1u, abort_flag, p.err, p.wait_ns);
     have_o = __all_sync(0xffffffffu, have_o);  // the TMEM loads below are warp-wide
     ptx::tc_fence_after();
-    // All UMMAs and TMA copies of this CTA have completed: the K ring is free to hold the partial result.
-    // Rows 64-127 of the accumulator (the remainders' share) go to the buffer first, rows 0-63 are added to them.
+    // All UMMAs and TMA copies of this CTA have completed: the rings are free to hold the partial result.
     ptx::named_bar_sync(1, kSoftmaxThreads);
     float* x = xbuf + row * kXRow + sub * 64;
-    if (quad >= 2) {
+    if constexpr (kWide) {
+      // every TMEM lane is a tree row of its own: its 64 columns go straight to the buffer
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float v[16];
@@ -457,29 +485,52 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
         for (int k = 0; k < 4; ++k) dst[k] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
       }
-    }
-    s_lsum[(quad >> 1) * 2 + sub][row] = l_run;
-    ptx::named_bar_sync(1, kSoftmaxThreads);
-    if (quad < 2) {
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float v[16];
-        if (have_o) {
-          ptx::tmem_ld16(o_cols + 16 * c, v);
-        } else {
-#pragma unroll
-          for (int k = 0; k < 16; ++k) v[k] = 0.f;
-        }
-        float4* dst = reinterpret_cast<float4*>(x + 16 * c);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float4 lo = dst[k];
-          dst[k] = make_float4(v[4 * k] + lo.x, v[4 * k + 1] + lo.y, v[4 * k + 2] + lo.z, v[4 * k + 3] + lo.w);
-        }
-      }
+      s_lsum[sub][row] = l_run;
+      ptx::named_bar_sync(1, kSoftmaxThreads);
       if (sub == 0) {   // the row's reference and the sum of its weights ride behind its 128 outputs
         xbuf[row * kXRow + kD] = m_ref;
-        xbuf[row * kXRow + kD + 1] = s_lsum[0][row] + s_lsum[1][row] + s_lsum[2][row] + s_lsum[3][row];
+        xbuf[row * kXRow + kD + 1] = s_lsum[0][row] + s_lsum[1][row];
+      }
+    } else {
+      // Rows 64-127 of the accumulator (the remainders' share) go to the buffer first, rows 0-63 are added to them.
+      if (quad >= 2) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[16];
+          if (have_o) {
+            ptx::tmem_ld16(o_cols + 16 * c, v);
+          } else {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) v[k] = 0.f;
+          }
+          float4* dst = reinterpret_cast<float4*>(x + 16 * c);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) dst[k] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+        }
+      }
+      s_lsum[(quad >> 1) * 2 + sub][row] = l_run;
+      ptx::named_bar_sync(1, kSoftmaxThreads);
+      if (quad < 2) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float v[16];
+          if (have_o) {
+            ptx::tmem_ld16(o_cols + 16 * c, v);
+          } else {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) v[k] = 0.f;
+          }
+          float4* dst = reinterpret_cast<float4*>(x + 16 * c);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float4 lo = dst[k];
+            dst[k] = make_float4(v[4 * k] + lo.x, v[4 * k + 1] + lo.y, v[4 * k + 2] + lo.z, v[4 * k + 3] + lo.w);
+          }
+        }
+        if (sub == 0) {   // the row's reference and the sum of its weights ride behind its 128 outputs
+          xbuf[row * kXRow + kD] = m_ref;
+          xbuf[row * kXRow + kD + 1] = s_lsum[0][row] + s_lsum[1][row] + s_lsum[2][row] + s_lsum[3][row];
+        }
       }
     }
     ptx::tc_fence_before();
@@ -527,7 +578,7 @@ k_tree_attn_bf16(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::named_bar_sync(1, kSoftmaxThreads);
     // 16 pieces of 8 outputs per row; consecutive threads take consecutive pieces (rolled: run-once code)
 #pragma unroll 1
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kRowsPerBlock / 16; ++i) {
       const int idx = i * kSoftmaxThreads + (int)threadIdx.x, rw = idx >> 4, piece = idx & 15;
       const int jj = rb * kRowsPerBlock + rw;
       if (jj >= p.T) continue;
@@ -583,7 +634,9 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   a.T = T;
   a.Hq = sh.Hq;
   a.Hkv = sh.Hkv;
-  a.n_rb = cascade_detail::ceil_div(T, kRowsPerBlock);
+  const bool wide = T > kRowsNarrow;
+  const int rows_per_block = wide ? kRowsWide : kRowsNarrow;
+  a.n_rb = cascade_detail::ceil_div(T, rows_per_block);
   a.prefix_cap = prefix_cap;
   a.prefix_len = prefix_len;
   a.anc = tree->d_anc;
@@ -608,7 +661,7 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
 
   const uint64_t dq[4] = {(uint64_t)kD, (uint64_t)sh.Hq, (uint64_t)T, (uint64_t)R};
   const uint64_t sq[3] = {(uint64_t)kD, (uint64_t)sh.Hq * kD, (uint64_t)T * sh.Hq * kD};
-  const uint32_t bq[4] = {64, 1, kRowsPerBlock, 1};
+  const uint32_t bq[4] = {64, 1, 64, 1};  // 64 rows per load: the wide form fetches its 128 rows in two
   const uint64_t dt[4] = {(uint64_t)kD, (uint64_t)sh.Hkv, (uint64_t)T, (uint64_t)R};
   const uint64_t stt[3] = {(uint64_t)kD, (uint64_t)sh.Hkv * kD, (uint64_t)T * sh.Hkv * kD};
   const uint32_t bkv[4] = {64, 1, kTileKeys, 1};
@@ -626,7 +679,8 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   if (!mq || !mkt || !mvt || !mkp || !mvp) return CASCADE_ERR_CUDA;
   bool& configured = ctx->attn_configured;
   if (!configured) {
-    CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_tree_attn_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_tree_attn_bf16<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    CASCADE_CUDA_TRY(cudaFuncSetAttribute(k_tree_attn_bf16<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     configured = true;
   }
   cudaLaunchConfig_t cfg = {};
@@ -643,7 +697,10 @@ int launch_tree_attn_bf16(cascade_ctx* ctx, const cascade_tree* tree, const __nv
   cfg.numAttrs = 1;
   {
     KernelScope ks(ctx, K_TREE_ATTN, s);
-    CASCADE_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_tree_attn_bf16, *mq, *mkp, *mvp, *mkt, *mvt, a));
+    if (wide)
+      CASCADE_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_tree_attn_bf16<true>, *mq, *mkp, *mvp, *mkt, *mvt, a));
+    else
+      CASCADE_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_tree_attn_bf16<false>, *mq, *mkp, *mvp, *mkt, *mvt, a));
   }
   return CASCADE_OK;
 }
