@@ -113,6 +113,35 @@ def test_two_full_width_layers_each_against_the_checker_on_the_same_input():
     wl2.close()
 
 
+@pytest.mark.parametrize("nodes,prefix,sigma", [(16, 256, 0.3), (64, 1024, 0.1)])
+def test_sweep_cell_through_one_layer(nodes, prefix, sigma):
+    """Two cells of the batched sweep (8 prompts x CFG pair, 7B-shaped widths) as the benchmark runs them: through
+    one full-width decoder layer, every output element.  The 64-node cell has 1040 projection rows (nine row chunks),
+    the wide form of the attention (65 rows in one 128-row block) and the head's whole-item mode (520 rows)."""
+    w = synth.workload("sweep", tree=f"topk{nodes}", prefix_len=prefix, sigma=sigma)
+    wl = LayerWorkload(w, n_layers=1, keep_logits=True)
+    s = wl.run(0)
+    torch.cuda.synchronize()
+    wl.ctx.check()
+    h = s.host
+    ref = O.verify_step(h["embed"], h["layers"], h["gamma_final"], h["w_head"], h["tok"], wl.parent, h["k_prefix"],
+                        h["v_prefix"], h["prefix_len"], h["draft_p"], h["uniforms"], w.n_heads, w.head_dim, w.eps,
+                        w.rope_base, w.cfg_scale, 1.0, w.tau_pos, w.tau_seq, w.tvd_budget, kv_bf16=True)
+    hid_err = np.abs(s.out["hidden_out"].cpu().numpy() - ref["hidden"]).max()
+    assert hid_err < HIDDEN_TOL, hid_err
+    logits = s.out["logits"].cpu().numpy()
+    logit_err = np.abs(logits - ref["head"]["logits"]).max()
+    assert logit_err < LOGIT_TOL, logit_err
+    feat = s.out["feat"].cpu().numpy().astype(np.float64)
+    rows = [O.relaxed_accept(feat[b], logits[b], h["tok"][b], wl.parent, h["draft_p"][b], h["uniforms"][b], w.tau_pos,
+                             w.tau_seq, w.tvd_budget) for b in range(w.B)]
+    st = G.compare_decisions(wl.parent, rows, s.out["accept"].cpu().numpy(), s.out["path_nodes"].cpu().numpy(),
+                             s.out["path_len"].cpu().numpy(), cb.SELECT_LONGEST)
+    print(f"sweep cell {nodes} nodes, prefix {prefix}, sigma {sigma}, through one layer: hidden {hid_err:.2e}, logits "
+          f"{logit_err:.2e}, nodes compared {st['nodes_compared']}/{st['nodes']}, paths {s.out['path_len'].cpu().tolist()}")
+    wl.close()
+
+
 @pytest.mark.parametrize("B", [1, 2])
 def test_head_at_vocabulary_65536(B):
     """61 and 122 activation rows against a [65536, 4096] head: 512 vocabulary tiles x 32 K blocks over 148 CTAs, so
