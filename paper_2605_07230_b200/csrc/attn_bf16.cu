@@ -3,7 +3,9 @@
 // for sm_100a.  Memory-bound decode-style kernel: every key/value row is streamed from HBM once per
 // (CFG row, head) and shared by all tree rows.
 //
-// One CTA per (KV split, query head x 64-row block, CFG row); the splits of one unit form a thread-block cluster.
+// One CTA per (KV split, query head x row block, CFG row); the splits of one unit form a thread-block cluster.  What
+// follows describes row blocks of 64 tree rows (trees of up to 64 rows); larger trees take the wide form, row blocks
+// of 128 (see the kernel's template parameter).
 //   * two producer threads stream 128-key K tiles and V tiles (bf16, 128-byte swizzle) through their own
 //     rings (2 and 3 slots) and ask the L2 for the tiles after those;
 //   * one thread issues the tensor-core work: S = Q K^T (UMMA 128x128x128) into one of two TMEM score
