@@ -65,15 +65,28 @@ __global__ void __launch_bounds__(kNormThreads) k_final_norm_mix(const E* __rest
   auto load_pair = [&](int i, float* vc, float* vu) {
     load8(row_c + 8 * i, vc);
     load8(row_u + 8 * i, vu);
-    for (int s2 = 0; s2 < n_add; ++s2) {
-      const float* a0 = add + (size_t)s2 * add_stride + 8 * (size_t)i;
-      float t[8];
-      load8(a0 + m * h, t);
+    // three slices at a time: their loads are issued before the first is used (one L2 round trip per slice,
+    // nine in a row, was most of this kernel's time); added in slice order
+    for (int s0 = 0; s0 < n_add; s0 += 3) {
+      float tc[3][8], tu[3][8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) vc[e] += t[e];
-      load8(a0 + ((size_t)(B + b) * T + j) * h, t);
+      for (int q = 0; q < 3; ++q) {
+        if (s0 + q < n_add) {
+          const float* a0 = add + (size_t)(s0 + q) * add_stride + 8 * (size_t)i;
+          load8(a0 + m * h, tc[q]);
+          load8(a0 + ((size_t)(B + b) * T + j) * h, tu[q]);
+        } else {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) vu[e] += t[e];
+          for (int e = 0; e < 8; ++e) tc[q][e] = tu[q][e] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 3; ++q)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          vc[e] += tc[q][e];
+          vu[e] += tu[q][e];
+        }
     }
   };
 #pragma unroll

@@ -42,6 +42,29 @@ __device__ __forceinline__ void add4(float4& a, const float4 b) {
   a.z += b.z;
   a.w += b.w;
 }
+// v + slices[0] + slices[1] + ... in that order, `stride` floats apart.  The loads of four slices are issued before the
+// first of them is used: these kernels run few warps per SM, and one L2 round trip per slice (a dependent chain
+// of up to nine) was most of their time.
+__device__ __forceinline__ float4 add_slices(float4 v, const float* p, int n, long long stride) {
+  int s = 0;
+  for (; s + 4 <= n; s += 4) {
+    const float4 t0 = load4(p + (size_t)s * stride), t1 = load4(p + (size_t)(s + 1) * stride),
+                 t2 = load4(p + (size_t)(s + 2) * stride), t3 = load4(p + (size_t)(s + 3) * stride);
+    add4(v, t0);
+    add4(v, t1);
+    add4(v, t2);
+    add4(v, t3);
+  }
+  if (s + 2 <= n) {
+    const float4 t0 = load4(p + (size_t)s * stride), t1 = load4(p + (size_t)(s + 1) * stride);
+    add4(v, t0);
+    add4(v, t1);
+    s += 2;
+  }
+  if (s < n) add4(v, load4(p + (size_t)s * stride));
+  return v;
+}
+
 // four consecutive operand values of row m, columns k..k+3 (k a multiple of 4): fp32, or the bf16 pair in the
 // GEMM's staged layout
 __device__ __forceinline__ void put_operand4(__nv_bfloat16* op, const OperandLayout& lay, float* f32, int K, int m, int k,
@@ -90,8 +113,7 @@ __global__ void __launch_bounds__(kRowThreads) k_resid_norm(float* __restrict__ 
     if (er != nullptr) {
       v = load4(er + 4 * c);
     } else {
-      v = load4(xr + 4 * c);
-      for (int s = 0; s < n_slices; ++s) add4(v, load4(slices + (size_t)s * slice_stride + (size_t)m * h + 4 * c));
+      v = add_slices(load4(xr + 4 * c), slices + (size_t)m * h + 4 * c, n_slices, slice_stride);
     }
     return v;
   };
@@ -155,9 +177,7 @@ __global__ void __launch_bounds__(kRowThreads) k_rope_split(const float* __restr
   }
   __syncthreads();
   auto col4 = [&](int c) {
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < n_slices; ++s) add4(a, load4(slices + (size_t)s * slice_stride + m * n_cols + c));
-    return a;
+    return add_slices(make_float4(0.f, 0.f, 0.f, 0.f), slices + m * n_cols + c, n_slices, slice_stride);
   };
   auto store4 = [](E* dst, size_t i, const float4 a) {
     if constexpr (sizeof(E) == 2) {
@@ -220,10 +240,20 @@ __global__ void __launch_bounds__(kRowThreads) k_swiglu(const float* __restrict_
     // different numbers of pieces (looked up in the table the first threads made)
     const int n_g = map.balanced ? s_cnt[0][(4 * c) / map.tile_cols - t0g] : map.n_slices;
     const int n_u = map.balanced ? s_cnt[1][(ffn + 4 * c) / map.tile_cols - t0u] : map.n_slices;
-    for (int s = 0; s < max(n_g, n_u); ++s) {  // one loop: the gate and up loads of a slice go out together
-      const float* row = slices + (size_t)s * slice_stride + m * 2 * ffn;
-      if (s < n_g) add4(g, load4(row + 4 * c));
-      if (s < n_u) add4(u, load4(row + ffn + 4 * c));
+    // the gate and up loads of up to four slices go out together (a dependent round trip per slice otherwise)
+    for (int s0 = 0; s0 < max(n_g, n_u); s0 += 4) {
+      float4 tg[4], tu[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float* row = slices + (size_t)(s0 + i) * slice_stride + m * 2 * ffn;
+        tg[i] = s0 + i < n_g ? load4(row + 4 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        tu[i] = s0 + i < n_u ? load4(row + ffn + 4 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        add4(g, tg[i]);
+        add4(u, tu[i]);
+      }
     }
     put_operand4(a_op, lay, a_f32, ffn, (int)m, 4 * c,
                  make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
