@@ -461,6 +461,59 @@ def measure_step(name, args, dev, peaks, world, local, over=None, light=False):
     return res, wl, parent
 
 
+def attention_back_to_back(w, dev, peaks, launches_per_graph=8, replays=10):
+    """The tree-attention kernel alone, launched back to back: a CUDA graph of `launches_per_graph` calls of
+    cascade_tree_attn over rotating stand-alone inputs (q, K, V ~ N(0,1), more bytes than the L2 between reuses), timed
+    with CUDA events around `replays` replays.  An event pair around a single launch inside the step also times the
+    launch and drain of the stream (about 5 us); this figure is the kernel's average duration when launches follow
+    each other."""
+    import torch
+    from paper_2605_07230_b200 import binding as cb
+    parent = w.parent()
+    T = len(parent)
+    R, H, D, P = 2 * w.B, w.n_heads, w.head_dim, w.prefix_len
+    ctx = cb.Context(cb.BF16, w.B, T, max(P, 1), w.h, H, H, D, w.V, 0)
+    tree = cb.Tree(ctx, parent)
+    per_set = R * (P + T) * H * D * 4
+    n_sets = max(2, int(np.ceil(3 * 126e6 / per_set)))
+    gen = torch.Generator(device=dev).manual_seed(w.seed)
+    mk = lambda *shape: torch.randn(shape, generator=gen, device=dev).to(torch.bfloat16)
+    sets = [dict(q=mk(R, T, H, D), kp=mk(R, P, H, D), vp=mk(R, P, H, D), kt=mk(R, T, H, D), vt=mk(R, T, H, D),
+                 out=torch.zeros((R, T, H, D), dtype=torch.bfloat16, device=dev)) for _ in range(n_sets)]
+    plen = torch.full((R,), P, dtype=torch.int32, device=dev)
+
+    def run(i):
+        x = sets[i % n_sets]
+        cb.cascade_tree_attn(ctx, tree, x["q"], x["kp"], x["vp"], P, plen, x["kt"], x["vt"], x["out"], 1.0 / np.sqrt(D))
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(4):
+            run(i)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(launches_per_graph):
+                run(i)
+        for _ in range(3):
+            g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(replays):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    ctx.check()
+    us = 1e3 * e0.elapsed_time(e1) / (replays * launches_per_graph)
+    nbytes = per_set + 2 * R * T * H * D * 2
+    tree.close()
+    ctx.close()
+    return {"us_per_launch": us, "launches": replays * launches_per_graph, "algorithmic_bytes": nbytes,
+            "achieved_gbs": nbytes / us / 1e3, "frac_of_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
+            "peak_source": peaks["source"], "inputs": f"{n_sets} rotating sets of {per_set / 1e6:.0f} MB, stand-alone q/K/V"}
+
+
 def accepted_length_table(dev, steps=8):
     """What the acceptance rule does on the Janus-shaped step: mean accepted drafts per step for three cluster
     tightnesses of the codebook, with the relaxation on (Eq. 1 + Eq. 2 sets) and off (plain Algorithm 1 test)."""
@@ -721,6 +774,8 @@ def main():
             wl.close()
             del wl
             torch.cuda.empty_cache()
+            if args.mode == "layer" and rank == 0 and synth.workload(name).dtype == "bf16":
+                res["tree_attn_back_to_back"] = attention_back_to_back(synth.workload(name), dev, peaks)
             if i == 0:
                 line = {"metric": METRIC, "value": res.pop("value"), "unit": UNIT, "n_gpus": world, "steps": res.pop("steps"),
                         "warmup": res.pop("warmup"), "ms_per_step": res.pop("ms_per_step"), "higher_is_better": True,
