@@ -41,7 +41,7 @@ NCU_TRAFFIC = {
     "janus": {"gemm_qkv": 108145664, "tree_attn": 15632384, "gemm_o": 35681792, "gemm_gate_up": 190507264, "gemm_down": 100555520, "gemm_head": 139249664},
     "lumina": {"gemm_qkv": 107926272, "tree_attn": 86904320, "gemm_o": 35683072, "gemm_gate_up": 190346752, "gemm_down": 100851456, "gemm_head": 544933632},
 }
-NCU_TRAFFIC_SOURCES = {"gemm_tc.cu": "3bbc44bff5fc1692", "attn_bf16.cu": "4feadd6018bb3218"}
+NCU_TRAFFIC_SOURCES = {"gemm_tc.cu": "3bbc44bff5fc1692", "attn_bf16.cu": "729009871e987da3"}
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
